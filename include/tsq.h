@@ -1,0 +1,165 @@
+/*
+ * tsq — threshold splitting (TS) + token-wise adaptive bit quantisation (TAB-Q) of an LLM
+ * split-point hidden state, on one NVIDIA B200 (sm_100a).
+ *
+ * Method: "Memory- and Latency-Constrained Inference of Large Language Models via Adaptive
+ * Split Computing", Sec. II-C.  Encode = Eq. "ts" (outliers with |x| >= tau leave, undistorted,
+ * as a CSR list) followed, per token row, by Algorithm 1 (TAB-Q) built on Eq. "Proposed" (AIQ):
+ * a per-token min/max range over the magnitudes, a per-token bit-width chosen from a candidate
+ * list by the distortion test, and the codes packed into word-aligned bit-planes.  Decode =
+ * Eq. "dequnt": unpack, (code + zero-point) * scale, outliers written back.
+ *
+ * Conventions for every call:
+ *  - plain C ABI; every pointer is marked HOST or DEVICE; the caller owns every buffer;
+ *  - tsq_encode / tsq_decode only enqueue work on `cuda_stream` (a cudaStream_t passed as
+ *    void*, NULL = the default stream): they never synchronise, allocate or copy to the host;
+ *  - errors are return values.  Conditions that only the GPU can see (outlier capacity
+ *    exceeded, malformed blob, a bounded wait that ran out) are recorded in the blob header's
+ *    `status` (encode) and in the workspace (encode and decode) and are read with
+ *    tsq_blob_info / tsq_workspace_status;
+ *  - device tensors are contiguous row-major [tokens x hidden], 16-bit elements, base address
+ *    16-byte aligned;
+ *  - arithmetic is IEEE binary32, round-to-nearest-even, true division semantics, no
+ *    flush-to-zero: results are bit-identical to a scalar evaluation of the paper's formulas.
+ */
+#ifndef TSQ_H_
+#define TSQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tsq_plan tsq_plan_t; /* opaque; host-owned; immutable after creation; may be shared by threads */
+
+typedef enum {
+  TSQ_OK = 0,
+  TSQ_ERR_INVALID_ARG = 1,
+  TSQ_ERR_UNSUPPORTED = 2,      /* legal for the method, declined by the GPU path (e.g. hidden % 8 != 0) */
+  TSQ_ERR_BUFFER_TOO_SMALL = 3,
+  TSQ_ERR_CUDA = 4,             /* a CUDA runtime call failed */
+  TSQ_ERR_CORRUPT_BLOB = 5,
+  TSQ_ERR_OUTLIER_OVERFLOW = 6, /* more outliers than the plan's capacity; the excess was dropped */
+  TSQ_ERR_TIMEOUT = 7           /* a bounded device-side wait ran out; re-initialise the workspace */
+} tsq_status_t;
+
+typedef enum { TSQ_F16 = 0, TSQ_BF16 = 1 } tsq_dtype_t;
+
+typedef struct {
+  size_t blob_bytes;      /* bytes of the blob buffer for `tokens` rows (capacity, not payload) */
+  size_t workspace_bytes; /* bytes of the workspace the plan needs (independent of `tokens`) */
+} tsq_sizes_t;
+
+typedef struct {
+  uint32_t status;        /* tsq_status_t recorded by the encoder */
+  uint32_t tokens, hidden, dtype;
+  uint64_t total_words;   /* 32-bit words of bit-planes in use */
+  uint64_t total_outliers;
+  uint64_t payload_bytes; /* bytes a sender would transmit: header + per-token fields + planes + CSR */
+} tsq_info_t;
+
+/*
+ * Blob format "TSQ1" (little endian; every section starts on a 16-byte boundary; capacities are
+ * those of the call's `tokens` and the plan; only the first total_words / total_outliers entries
+ * of the last two sections are meaningful).  WPP = ceil(hidden / 32).
+ *
+ *   header   64 B  u32 magic 'TSQ1' | u32 version=1 | u32 dtype | u32 hidden | u32 tokens |
+ *                  u32 n_bits | u8 bits[8] | f32 tau | f32 delta | u64 total_words |
+ *                  u64 total_outliers | u32 status | u32 outlier_capacity
+ *   bits     u8  [tokens]      chosen bit-width b* (1 sign bit + (b*-1)-bit magnitude code)
+ *   scale    f32 [tokens]      AIQ scale s
+ *   zp       i32 [tokens]      AIQ zero-point, restore = (code + zp) * s
+ *   word_off u32 [tokens+1]    exclusive prefix sum of b* x WPP
+ *   out_ptr  u32 [tokens+1]    CSR row pointers (exclusive prefix sum of per-token outlier counts)
+ *   words    u32 [tokens x bmax x WPP]  token t owns b* planes of WPP words from word_off[t]:
+ *                  plane 0 = sign bits of the inliers, plane 1+k = bit k of the magnitude codes;
+ *                  bit i of word w belongs to element 32*w + i; pad bits are 0
+ *   outl     u32 [outlier_capacity]     (column << 16) | original 16-bit pattern, columns ascending
+ */
+
+/*
+ * Create a plan: parameters of TS (tau, Eq. "ts") and of TAB-Q (candidate bit-widths and the
+ * distortion tolerance delta of Algorithm 1; the paper's default is delta = 0.2).
+ *   out          HOST   receives the plan; destroy with tsq_plan_destroy
+ *   device              CUDA device ordinal the plan's kernels will run on
+ *   hidden              row length H, 8 <= H <= 65536, H % 8 == 0 (else TSQ_ERR_UNSUPPORTED)
+ *   max_tokens          largest `tokens` any call will pass (>= 0); tokens * H < 2^32 and
+ *                       tokens * bmax * WPP < 2^32
+ *   tau                 threshold; |x| >= tau, NaN and +-Inf become outliers.  +INF disables TS
+ *                       for finite values, tau <= 0 makes every element an outlier.  NaN is invalid
+ *   bits         HOST   n_bits strictly increasing candidates, each in [2, 8]; 1 <= n_bits <= 7
+ *   delta               tolerance on the mean absolute code distortion (may be negative: no
+ *                       lower candidate is ever accepted)
+ *   max_outliers        CSR capacity in entries; 0 = worst case tokens * H
+ * Queries device attributes; allocates no device memory.
+ */
+tsq_status_t tsq_plan(tsq_plan_t **out, int device, tsq_dtype_t dtype, int32_t hidden, int64_t max_tokens,
+                      float tau, const int32_t *bits, int32_t n_bits, float delta, int64_t max_outliers);
+
+/* Buffer sizes for a call with `tokens` rows (0 <= tokens <= max_tokens). `out` is HOST. */
+tsq_status_t tsq_plan_sizes(const tsq_plan_t *plan, int64_t tokens, tsq_sizes_t *out);
+
+/*
+ * Zero a workspace (DEVICE, workspace_bytes, 16-byte aligned) on `cuda_stream`.  Required once
+ * before the buffer's first use and after any TSQ_ERR_TIMEOUT; encode and decode leave it ready
+ * for the next call.  One workspace serves one call at a time: calls that may overlap on the GPU
+ * need separate workspaces.  (Variable-length placement, the prefix sums behind word_off and
+ * out_ptr, is resolved inside the encode kernel through this buffer.)
+ */
+tsq_status_t tsq_workspace_init(const tsq_plan_t *plan, void *ws_dev, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Encode x (DEVICE, [tokens x hidden]) into blob (DEVICE, >= blob_bytes from tsq_plan_sizes,
+ * 16-byte aligned): TS (Eq. "ts") + TAB-Q (Algorithm 1, token-wise) + bit-plane packing, one
+ * kernel launch.  tokens == 0 writes an empty, valid blob.  Returns argument errors before
+ * anything is enqueued.
+ */
+tsq_status_t tsq_encode(const tsq_plan_t *plan, const void *x_dev, int64_t tokens, void *blob_dev,
+                        size_t blob_bytes, void *ws_dev, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Decode blob (DEVICE) into y (DEVICE, [tokens x hidden]): Eq. "dequnt".  The kernel validates the
+ * header against the plan and `tokens`, and every per-token field against the blob's capacities,
+ * before using it; on a mismatch it writes nothing for that blob/row and records
+ * TSQ_ERR_CORRUPT_BLOB (or the encoder's own non-zero status) in the workspace.
+ */
+tsq_status_t tsq_decode(const tsq_plan_t *plan, const void *blob_dev, size_t blob_bytes, int64_t tokens,
+                        void *y_dev, void *ws_dev, size_t ws_bytes, void *cuda_stream);
+
+/* Copy the blob's header to the host and summarise it. Synchronises `cuda_stream`. `out` is HOST. */
+tsq_status_t tsq_blob_info(const void *blob_dev, tsq_info_t *out, void *cuda_stream);
+
+/*
+ * First asynchronous error recorded in the workspace since it was initialised (TSQ_OK if none),
+ * for the encoder and for the decoder.  Synchronises `cuda_stream`.  Both outputs are HOST.
+ */
+tsq_status_t tsq_workspace_status(const void *ws_dev, uint32_t *encode_status, uint32_t *decode_status,
+                                  void *cuda_stream);
+
+/*
+ * Host-buffer convenience calls (x_host / blob_host / y_host are HOST, ideally pinned; the *_dev
+ * staging buffers are DEVICE and caller-owned, sized as for tsq_encode / tsq_decode).
+ * tsq_encode_host copies x to the device, encodes, and copies back the header, the per-token
+ * fields and only the used part of the planes and of the CSR list; *payload_bytes (HOST) receives
+ * the number of meaningful bytes.  tsq_decode_host copies a blob produced that way to the device,
+ * decodes and copies y back.  Both synchronise `cuda_stream` and return the asynchronous status.
+ */
+tsq_status_t tsq_encode_host(const tsq_plan_t *plan, const void *x_host, int64_t tokens, void *blob_host,
+                             size_t blob_bytes, uint64_t *payload_bytes, void *x_dev, void *blob_dev,
+                             void *ws_dev, size_t ws_bytes, void *cuda_stream);
+tsq_status_t tsq_decode_host(const tsq_plan_t *plan, const void *blob_host, size_t blob_bytes, int64_t tokens,
+                             void *y_host, void *blob_dev, void *y_dev, void *ws_dev, size_t ws_bytes,
+                             void *cuda_stream);
+
+/* Number of kernels the library has launched in this process (all plans, all streams). */
+uint64_t tsq_kernel_launch_count(void);
+
+void tsq_plan_destroy(tsq_plan_t *plan);
+const char *tsq_status_string(tsq_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSQ_H_ */

@@ -1,0 +1,360 @@
+// Host side of the tsq C ABI: plan creation, buffer sizing, argument checks, launches.
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "tsq_internal.h"
+
+namespace tsq {
+namespace {
+
+std::atomic<unsigned long long> g_launches{0};
+
+// Value of a non-negative 16-bit pattern, on the host (used once per plan, for the threshold).
+float pattern_value(tsq_dtype_t dtype, uint32_t pat) {
+  if (dtype == TSQ_BF16) {
+    const uint32_t u = pat << 16;
+    float f;
+    std::memcpy(&f, &u, 4);
+    return f;
+  }
+  const int e = (pat >> 10) & 0x1f;
+  const int frac = pat & 0x3ff;
+  if (e == 0x1f) return frac ? NAN : INFINITY;
+  if (e == 0) return std::ldexp(static_cast<float>(frac), -24);
+  return std::ldexp(static_cast<float>(frac | 0x400), e - 25);
+}
+
+// Smallest non-negative 16-bit pattern whose value is >= tau (tau is not NaN).  Patterns of
+// non-negative values are ordered like the values, so a bisection over [0, +Inf pattern] finds it.
+uint32_t threshold_pattern(tsq_dtype_t dtype, float tau) {
+  const uint32_t inf_pat = dtype == TSQ_BF16 ? 0x7f80u : 0x7c00u;
+  if (tau <= 0.0f) return 0u;
+  uint32_t lo = 0u, hi = inf_pat;  // invariant: value(hi) >= tau
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi) / 2u;
+    if (pattern_value(dtype, mid) >= tau) {
+      hi = mid;
+    } else {
+      lo = mid + 1u;
+    }
+  }
+  return hi;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+__global__ void workspace_init_kernel(WsControl* ws, uint32_t desc_capacity) { ws->desc_capacity = desc_capacity; }
+
+}  // namespace
+}  // namespace tsq
+
+struct tsq_plan {
+  int device;
+  tsq_dtype_t dtype;
+  uint32_t hidden, units, chunks, row_bytes;
+  unsigned long long max_tokens, max_outliers;
+  float tau, delta;
+  int32_t n_bits;
+  int32_t bits[8];
+  int32_t bmax;
+  int32_t s_max;
+  uint32_t thr16;
+  int threads;
+  uint32_t stages;
+  size_t enc_smem, dec_smem;
+  int enc_grid_limit;  // CTAs that are co-resident on the device
+  size_t workspace_bytes;
+};
+
+using namespace tsq;
+
+extern "C" {
+
+const char* tsq_status_string(tsq_status_t status) {
+  switch (status) {
+    case TSQ_OK: return "ok";
+    case TSQ_ERR_INVALID_ARG: return "invalid argument";
+    case TSQ_ERR_UNSUPPORTED: return "unsupported by the GPU path";
+    case TSQ_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case TSQ_ERR_CUDA: return "CUDA runtime error";
+    case TSQ_ERR_CORRUPT_BLOB: return "corrupt blob";
+    case TSQ_ERR_OUTLIER_OVERFLOW: return "outlier capacity exceeded";
+    case TSQ_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+uint64_t tsq_kernel_launch_count(void) { return g_launches.load(); }
+
+tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t hidden, int64_t max_tokens, float tau,
+                      const int32_t* bits, int32_t n_bits, float delta, int64_t max_outliers) {
+  if (!out) return TSQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (dtype != TSQ_F16 && dtype != TSQ_BF16) return TSQ_ERR_INVALID_ARG;
+  if (!bits || n_bits < 1 || n_bits > kMaxCand) return TSQ_ERR_INVALID_ARG;
+  for (int i = 0; i < n_bits; ++i) {
+    if (bits[i] < 2 || bits[i] > 8) return TSQ_ERR_INVALID_ARG;
+    if (i > 0 && bits[i] <= bits[i - 1]) return TSQ_ERR_INVALID_ARG;
+  }
+  if (tau != tau || delta != delta) return TSQ_ERR_INVALID_ARG;
+  if (hidden < 1 || hidden > 65536 || max_tokens < 0 || max_outliers < 0 || device < 0) return TSQ_ERR_INVALID_ARG;
+  if (hidden % 8 != 0) return TSQ_ERR_UNSUPPORTED;
+  const unsigned long long T = static_cast<unsigned long long>(max_tokens), H = static_cast<unsigned long long>(hidden);
+  const int bmax = bits[n_bits - 1];
+  const unsigned long long wpp = (H + 31) / 32;
+  if (T * H >= (1ull << 32) || T * bmax * wpp >= (1ull << 32)) return TSQ_ERR_INVALID_ARG;
+
+  tsq_plan_t* p = new (std::nothrow) tsq_plan_t();
+  if (!p) return TSQ_ERR_INVALID_ARG;
+  p->device = device;
+  p->dtype = dtype;
+  p->hidden = static_cast<uint32_t>(hidden);
+  p->units = static_cast<uint32_t>(wpp);
+  p->chunks = static_cast<uint32_t>(hidden / 8);
+  p->row_bytes = static_cast<uint32_t>(hidden) * 2u;
+  p->max_tokens = T;
+  p->max_outliers = static_cast<unsigned long long>(max_outliers);
+  p->tau = tau;
+  p->delta = delta;
+  p->n_bits = n_bits;
+  for (int i = 0; i < 8; ++i) p->bits[i] = i < n_bits ? bits[i] : 0;
+  p->bmax = bmax;
+  const double smax = std::floor(static_cast<double>(delta) * static_cast<double>(hidden));
+  p->s_max = smax < -1.0 ? -1 : (smax > 2147483647.0 ? 2147483647 : static_cast<int32_t>(smax));
+  p->thr16 = threshold_pattern(dtype, tau);
+  p->threads = static_cast<int>(((p->units + 31u) / 32u) * 32u);
+  if (p->threads > kMaxThreads) p->threads = kMaxThreads;
+  const size_t row_stride = (static_cast<size_t>(p->row_bytes) + 127u) & ~static_cast<size_t>(127u);
+  size_t stages = (54u * 1024u) / row_stride;
+  if (stages < 1) stages = 1;
+  if (stages > static_cast<size_t>(kMaxStages)) stages = kMaxStages;
+  p->stages = static_cast<uint32_t>(stages);
+  p->enc_smem = encode_smem_bytes(p->units, p->row_bytes, p->stages);
+  p->dec_smem = decode_smem_bytes(p->row_bytes);
+  const unsigned long long desc = T > 0 ? T : 1;
+  p->workspace_bytes = sizeof(WsControl) + 2 * sizeof(unsigned long long) * desc;
+
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) {
+    delete p;
+    return TSQ_ERR_CUDA;
+  }
+  int prev_dev = 0;
+  cudaGetDevice(&prev_dev);
+  bool ok = cudaSetDevice(device) == cudaSuccess;
+  int sms = 0, enc_blocks = 0, dec_blocks = 0;
+  ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess;
+  ok = ok && encode_kernel_attrs(dtype == TSQ_BF16, p->threads, p->enc_smem, &enc_blocks) == cudaSuccess;
+  ok = ok && decode_kernel_attrs(dtype == TSQ_BF16, p->threads, p->dec_smem, &dec_blocks) == cudaSuccess;
+  cudaSetDevice(prev_dev);
+  if (!ok || enc_blocks < 1 || dec_blocks < 1 || sms < 1) {
+    cudaGetLastError();
+    delete p;
+    return TSQ_ERR_CUDA;
+  }
+  p->enc_grid_limit = enc_blocks * sms;
+  *out = p;
+  return TSQ_OK;
+}
+
+void tsq_plan_destroy(tsq_plan_t* plan) { delete plan; }
+
+static BlobLayout layout_for(const tsq_plan_t* plan, unsigned long long tokens) {
+  unsigned long long cap = tokens * plan->hidden;
+  if (plan->max_outliers > 0 && plan->max_outliers < cap) cap = plan->max_outliers;
+  return make_layout(plan->hidden, tokens, static_cast<uint32_t>(plan->bmax), cap);
+}
+
+tsq_status_t tsq_plan_sizes(const tsq_plan_t* plan, int64_t tokens, tsq_sizes_t* out) {
+  if (!plan || !out || tokens < 0 || static_cast<unsigned long long>(tokens) > plan->max_tokens) return TSQ_ERR_INVALID_ARG;
+  const BlobLayout L = layout_for(plan, static_cast<unsigned long long>(tokens));
+  out->blob_bytes = static_cast<size_t>(L.total);
+  out->workspace_bytes = plan->workspace_bytes;
+  return TSQ_OK;
+}
+
+tsq_status_t tsq_workspace_init(const tsq_plan_t* plan, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  if (!plan || !ws_dev || !aligned16(ws_dev)) return TSQ_ERR_INVALID_ARG;
+  if (ws_bytes < plan->workspace_bytes) return TSQ_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(ws_dev, 0, plan->workspace_bytes, st) != cudaSuccess) return TSQ_ERR_CUDA;
+  const uint32_t cap = static_cast<uint32_t>((plan->workspace_bytes - sizeof(WsControl)) / (2 * sizeof(unsigned long long)));
+  workspace_init_kernel<<<1, 1, 0, st>>>(static_cast<WsControl*>(ws_dev), cap);
+  g_launches.fetch_add(1);
+  return cudaGetLastError() == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
+}
+
+tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t tokens, void* blob_dev, size_t blob_bytes,
+                        void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  if (!plan || !blob_dev || !ws_dev || tokens < 0 || static_cast<unsigned long long>(tokens) > plan->max_tokens)
+    return TSQ_ERR_INVALID_ARG;
+  if (tokens > 0 && !x_dev) return TSQ_ERR_INVALID_ARG;
+  if (!aligned16(x_dev) || !aligned16(blob_dev) || !aligned16(ws_dev)) return TSQ_ERR_INVALID_ARG;
+  const BlobLayout L = layout_for(plan, static_cast<unsigned long long>(tokens));
+  if (blob_bytes < L.total || ws_bytes < plan->workspace_bytes) return TSQ_ERR_BUFFER_TOO_SMALL;
+
+  EncodeParams p;
+  std::memset(&p, 0, sizeof p);
+  p.x = static_cast<const uint16_t*>(x_dev);
+  p.blob = static_cast<unsigned char*>(blob_dev);
+  p.ws = static_cast<WsControl*>(ws_dev);
+  const unsigned long long desc = plan->max_tokens > 0 ? plan->max_tokens : 1;
+  p.desc_words = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(ws_dev) + sizeof(WsControl));
+  p.desc_outl = p.desc_words + desc;
+  p.lay = L;
+  p.tokens = static_cast<uint32_t>(tokens);
+  p.hidden = plan->hidden;
+  p.units = plan->units;
+  p.chunks = plan->chunks;
+  p.thr16 = plan->thr16;
+  p.n_bits = plan->n_bits;
+  for (int i = 0; i < 8; ++i) p.bits[i] = plan->bits[i];
+  p.s_max = plan->s_max;
+  p.stages = plan->stages;
+  p.row_bytes = plan->row_bytes;
+  p.dtype = static_cast<uint32_t>(plan->dtype);
+  p.tau = plan->tau;
+  p.delta = plan->delta;
+
+  int grid = tokens < plan->enc_grid_limit ? static_cast<int>(tokens) : plan->enc_grid_limit;
+  if (grid < 1) grid = 1;
+  const cudaError_t e = launch_encode(p, grid, plan->threads, plan->enc_smem, static_cast<cudaStream_t>(cuda_stream));
+  g_launches.fetch_add(1);
+  return e == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
+}
+
+tsq_status_t tsq_decode(const tsq_plan_t* plan, const void* blob_dev, size_t blob_bytes, int64_t tokens, void* y_dev,
+                        void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  if (!plan || !blob_dev || !ws_dev || tokens < 0 || static_cast<unsigned long long>(tokens) > plan->max_tokens)
+    return TSQ_ERR_INVALID_ARG;
+  if (tokens > 0 && !y_dev) return TSQ_ERR_INVALID_ARG;
+  if (!aligned16(y_dev) || !aligned16(blob_dev) || !aligned16(ws_dev)) return TSQ_ERR_INVALID_ARG;
+  const BlobLayout L = layout_for(plan, static_cast<unsigned long long>(tokens));
+  if (blob_bytes < L.total || ws_bytes < plan->workspace_bytes) return TSQ_ERR_BUFFER_TOO_SMALL;
+  if (tokens == 0) return TSQ_OK;
+
+  DecodeParams p;
+  std::memset(&p, 0, sizeof p);
+  p.blob = static_cast<const unsigned char*>(blob_dev);
+  p.y = static_cast<uint16_t*>(y_dev);
+  p.ws = static_cast<WsControl*>(ws_dev);
+  p.lay = L;
+  p.tokens = static_cast<uint32_t>(tokens);
+  p.hidden = plan->hidden;
+  p.units = plan->units;
+  p.chunks = plan->chunks;
+  p.bmax = static_cast<uint32_t>(plan->bmax);
+  p.dtype = static_cast<uint32_t>(plan->dtype);
+  p.blob_bytes = blob_bytes;
+  const cudaError_t e = launch_decode(p, static_cast<int>(tokens), plan->threads, plan->dec_smem,
+                                      static_cast<cudaStream_t>(cuda_stream));
+  g_launches.fetch_add(1);
+  return e == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
+}
+
+static unsigned long long payload_of(unsigned long long tokens, unsigned long long words, unsigned long long outliers) {
+  return 64ull + 9ull * tokens + 8ull * (tokens + 1ull) + 4ull * words + 4ull * outliers;
+}
+
+tsq_status_t tsq_blob_info(const void* blob_dev, tsq_info_t* out, void* cuda_stream) {
+  if (!blob_dev || !out) return TSQ_ERR_INVALID_ARG;
+  BlobHeader h;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(&h, blob_dev, sizeof h, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TSQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TSQ_ERR_CUDA;
+  if (h.magic != kMagic || h.version != kVersion) return TSQ_ERR_CORRUPT_BLOB;
+  out->status = h.status;
+  out->tokens = h.tokens;
+  out->hidden = h.hidden;
+  out->dtype = h.dtype;
+  out->total_words = h.total_words;
+  out->total_outliers = h.total_outliers;
+  const unsigned long long stored = h.total_outliers < h.outlier_capacity ? h.total_outliers : h.outlier_capacity;
+  out->payload_bytes = payload_of(h.tokens, h.total_words, stored);
+  return TSQ_OK;
+}
+
+tsq_status_t tsq_workspace_status(const void* ws_dev, uint32_t* encode_status, uint32_t* decode_status,
+                                  void* cuda_stream) {
+  if (!ws_dev) return TSQ_ERR_INVALID_ARG;
+  WsControl c;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(&c, ws_dev, sizeof c, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TSQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TSQ_ERR_CUDA;
+  if (encode_status) *encode_status = c.enc_status;
+  if (decode_status) *decode_status = c.dec_status;
+  return TSQ_OK;
+}
+
+tsq_status_t tsq_encode_host(const tsq_plan_t* plan, const void* x_host, int64_t tokens, void* blob_host,
+                             size_t blob_bytes, uint64_t* payload_bytes, void* x_dev, void* blob_dev, void* ws_dev,
+                             size_t ws_bytes, void* cuda_stream) {
+  if (!plan || !blob_host || !blob_dev || !ws_dev || tokens < 0) return TSQ_ERR_INVALID_ARG;
+  if (tokens > 0 && (!x_host || !x_dev)) return TSQ_ERR_INVALID_ARG;
+  if (static_cast<unsigned long long>(tokens) > plan->max_tokens) return TSQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const BlobLayout L = layout_for(plan, static_cast<unsigned long long>(tokens));
+  if (blob_bytes < L.total) return TSQ_ERR_BUFFER_TOO_SMALL;
+  const size_t x_bytes = static_cast<size_t>(tokens) * plan->hidden * 2u;
+  if (x_bytes && cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TSQ_ERR_CUDA;
+  const tsq_status_t s = tsq_encode(plan, x_dev, tokens, blob_dev, blob_bytes, ws_dev, ws_bytes, cuda_stream);
+  if (s != TSQ_OK) return s;
+  // header and per-token fields first: they say how much of the planes and of the CSR list is in use
+  unsigned char* bh = static_cast<unsigned char*>(blob_host);
+  const unsigned char* bd = static_cast<const unsigned char*>(blob_dev);
+  if (cudaMemcpyAsync(bh, bd, static_cast<size_t>(L.off_words), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TSQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TSQ_ERR_CUDA;
+  BlobHeader h;
+  std::memcpy(&h, bh, sizeof h);
+  if (h.magic != kMagic) return TSQ_ERR_CORRUPT_BLOB;
+  const unsigned long long stored = h.total_outliers < L.outlier_capacity ? h.total_outliers : L.outlier_capacity;
+  if (h.total_words > L.words_capacity) return TSQ_ERR_CORRUPT_BLOB;
+  if (h.total_words && cudaMemcpyAsync(bh + L.off_words, bd + L.off_words, static_cast<size_t>(4 * h.total_words),
+                                       cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return TSQ_ERR_CUDA;
+  if (stored && cudaMemcpyAsync(bh + L.off_outl, bd + L.off_outl, static_cast<size_t>(4 * stored), cudaMemcpyDeviceToHost,
+                                st) != cudaSuccess)
+    return TSQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TSQ_ERR_CUDA;
+  if (payload_bytes) *payload_bytes = payload_of(h.tokens, h.total_words, stored);
+  return static_cast<tsq_status_t>(h.status);
+}
+
+tsq_status_t tsq_decode_host(const tsq_plan_t* plan, const void* blob_host, size_t blob_bytes, int64_t tokens,
+                             void* y_host, void* blob_dev, void* y_dev, void* ws_dev, size_t ws_bytes,
+                             void* cuda_stream) {
+  if (!plan || !blob_host || !blob_dev || !ws_dev || tokens < 0) return TSQ_ERR_INVALID_ARG;
+  if (tokens > 0 && (!y_host || !y_dev)) return TSQ_ERR_INVALID_ARG;
+  if (static_cast<unsigned long long>(tokens) > plan->max_tokens) return TSQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const BlobLayout L = layout_for(plan, static_cast<unsigned long long>(tokens));
+  if (blob_bytes < L.total) return TSQ_ERR_BUFFER_TOO_SMALL;
+  BlobHeader h;
+  std::memcpy(&h, blob_host, sizeof h);
+  if (h.magic != kMagic || h.version != kVersion || h.tokens != static_cast<uint32_t>(tokens) ||
+      h.total_words > L.words_capacity)
+    return TSQ_ERR_CORRUPT_BLOB;
+  const unsigned long long stored = h.total_outliers < L.outlier_capacity ? h.total_outliers : L.outlier_capacity;
+  const unsigned char* bh = static_cast<const unsigned char*>(blob_host);
+  unsigned char* bd = static_cast<unsigned char*>(blob_dev);
+  if (cudaMemcpyAsync(bd, bh, static_cast<size_t>(L.off_words), cudaMemcpyHostToDevice, st) != cudaSuccess) return TSQ_ERR_CUDA;
+  if (h.total_words && cudaMemcpyAsync(bd + L.off_words, bh + L.off_words, static_cast<size_t>(4 * h.total_words),
+                                       cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return TSQ_ERR_CUDA;
+  if (stored && cudaMemcpyAsync(bd + L.off_outl, bh + L.off_outl, static_cast<size_t>(4 * stored), cudaMemcpyHostToDevice,
+                                st) != cudaSuccess)
+    return TSQ_ERR_CUDA;
+  const tsq_status_t s = tsq_decode(plan, blob_dev, blob_bytes, tokens, y_dev, ws_dev, ws_bytes, cuda_stream);
+  if (s != TSQ_OK) return s;
+  const size_t y_bytes = static_cast<size_t>(tokens) * plan->hidden * 2u;
+  if (y_bytes && cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TSQ_ERR_CUDA;
+  uint32_t dec = 0;
+  const tsq_status_t ws = tsq_workspace_status(ws_dev, nullptr, &dec, cuda_stream);
+  if (ws != TSQ_OK) return ws;
+  return static_cast<tsq_status_t>(dec);
+}
+
+}  // extern "C"

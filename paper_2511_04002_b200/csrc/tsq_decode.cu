@@ -1,0 +1,167 @@
+// tsq decode kernel: Eq. "dequnt" — unpack the bit-planes of one token, restore
+// (code + zero-point) * scale, round once to the 16-bit type, put the sign back, then write the
+// outliers of T_above over their slots.  One CTA per token row; the row is assembled in shared
+// memory and leaves through one bulk asynchronous store.
+//
+// Every field read from the blob is checked against the capacities of the call before it is used
+// as an index: a malformed blob makes the kernel record TSQ_ERR_CORRUPT_BLOB and skip the row.
+
+#include "tsq_device.cuh"
+#include "tsq_internal.h"
+
+namespace tsq {
+namespace {
+
+constexpr float kTwo23 = 8388608.0f;
+constexpr uint32_t kTwo23Bits = 0x4B000000u;
+
+__device__ __forceinline__ void record_decode_error(const DecodeParams& p, uint32_t code) {
+  atomicCAS(&p.ws->dec_status, 0u, code);
+}
+
+
+// Unpack, dequantise and stage this thread's units of one row.
+//   DIRECT = false: float(code + zp) is formed without a conversion instruction: 2^23 + n carries
+//   n in its low mantissa bits, and (2^23 + n) * s - 2^23 * s equals n * s exactly, so one FMA
+//   rounds n * s once (2^23 * s is a power-of-two multiple of s, hence exact while finite).
+//   DIRECT = true: int -> float conversion and one multiplication.
+template <bool BF16, bool DIRECT>
+__device__ __forceinline__ void restore_units(const DecodeParams& p, const uint32_t* words, uint32_t b, float s,
+                                              int32_t zp) {
+  using E = Elem<BF16>;
+  extern __shared__ __align__(128) unsigned char smem_dyn[];
+  uint4* stage4 = reinterpret_cast<uint4*>(smem_dyn);
+  const float neg_bias = DIRECT ? 0.0f : -__fmul_rn(kTwo23, s);
+  const uint32_t int_bias = kTwo23Bits + static_cast<uint32_t>(zp);
+  for (uint32_t u = threadIdx.x; u < p.units; u += blockDim.x) {
+    uint32_t r[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      r[k] = (static_cast<uint32_t>(k) < b) ? __ldg(words + static_cast<size_t>(k) * p.lay.wpp + u) : 0u;
+    }
+    transpose8x32(r);  // r[i] byte c = (code << 1 | sign) of element 8c + i
+    const uint32_t rot = (u >> 1) & 3u;
+#pragma unroll
+    for (uint32_t j = 0; j < 4; ++j) {
+      const uint32_t cc = (j + rot) & 3u;
+      const uint32_t cidx = 4u * u + cc;
+      if (cidx >= p.chunks) continue;
+      const uint32_t shift = 8u * cc;
+      uint32_t out[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t blo = (r[2 * i] >> shift) & 0xffu, bhi = (r[2 * i + 1] >> shift) & 0xffu;
+        float flo, fhi;
+        if (DIRECT) {
+          flo = __fmul_rn(__int2float_rn(static_cast<int>(blo >> 1) + zp), s);
+          fhi = __fmul_rn(__int2float_rn(static_cast<int>(bhi >> 1) + zp), s);
+        } else {
+          flo = fmaf(__uint_as_float(int_bias + (blo >> 1)), s, neg_bias);
+          fhi = fmaf(__uint_as_float(int_bias + (bhi >> 1)), s, neg_bias);
+        }
+        out[i] = E::pack_rn(flo, fhi) | ((blo & 1u) << 15) | ((bhi & 1u) << 31);
+      }
+      stage4[cidx] = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+  }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kMaxThreads) decode_kernel(const DecodeParams p) {
+  extern __shared__ __align__(128) unsigned char smem_dyn[];  // one output row
+  const uint32_t tid = threadIdx.x;
+  const uint32_t t = blockIdx.x;
+
+  // ---- header against the plan and the call ----
+  const BlobHeader* h = reinterpret_cast<const BlobHeader*>(p.blob);
+  if (h->magic != kMagic || h->version != kVersion) {
+    if (tid == 0) record_decode_error(p, TSQ_ERR_CORRUPT_BLOB);
+    return;
+  }
+  if (h->status != TSQ_OK) {  // the encoder flagged this blob: pass its status on
+    if (tid == 0) record_decode_error(p, h->status);
+    return;
+  }
+  const bool header_ok = h->dtype == p.dtype && h->hidden == p.hidden && h->tokens == p.tokens && h->n_bits >= 1u &&
+                         h->n_bits <= static_cast<uint32_t>(kMaxCand) && h->bits[(h->n_bits - 1u) & 7u] == p.bmax &&
+                         h->outlier_capacity == static_cast<uint32_t>(p.lay.outlier_capacity) &&
+                         h->total_words <= p.lay.words_capacity && h->total_outliers <= p.lay.outlier_capacity;
+  if (!header_ok) {
+    if (tid == 0) record_decode_error(p, TSQ_ERR_CORRUPT_BLOB);
+    return;
+  }
+
+  // ---- this token's fields ----
+  const uint32_t b = reinterpret_cast<const uint8_t*>(p.blob + p.lay.off_bits)[t];
+  const float s = reinterpret_cast<const float*>(p.blob + p.lay.off_scale)[t];
+  const int32_t zp = reinterpret_cast<const int32_t*>(p.blob + p.lay.off_zp)[t];
+  const uint32_t wo = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_word_off)[t];
+  const uint32_t wo_next = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_word_off)[t + 1];
+  const uint32_t p0 = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_out_ptr)[t];
+  const uint32_t p1 = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_out_ptr)[t + 1];
+  const unsigned long long span = static_cast<unsigned long long>(b) * p.lay.wpp;
+  const bool row_ok = b >= 2u && b <= p.bmax && wo + span <= h->total_words && wo_next == wo + span && p0 <= p1 &&
+                      p1 <= h->total_outliers && (p1 - p0) <= p.hidden && zp >= 0 && zp < (1 << 22);
+  if (!row_ok) {
+    if (tid == 0) record_decode_error(p, TSQ_ERR_CORRUPT_BLOB);
+    return;
+  }
+
+  const uint32_t* words = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_words) + wo;
+  // 2^23 * s must stay finite for the conversion-free path; huge scales take the plain one.
+  if (s <= 0x1p100f) {
+    restore_units<BF16, false>(p, words, b, s, zp);
+  } else {
+    restore_units<BF16, true>(p, words, b, s, zp);
+  }
+  __syncthreads();
+
+  // ---- "+ T_above": each outlier slot decoded to +0, so adding equals overwriting ----
+  if (p1 != p0) {
+    const uint32_t* outl = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_outl);
+    uint16_t* stage16 = reinterpret_cast<uint16_t*>(smem_dyn);
+    bool bad = false;
+    for (uint32_t q = p0 + tid; q < p1; q += blockDim.x) {
+      const uint32_t e = __ldg(outl + q);
+      const uint32_t col = e >> 16;
+      if (col < p.hidden) {
+        stage16[col] = static_cast<uint16_t>(e & 0xffffu);
+      } else {
+        bad = true;
+      }
+    }
+    if (bad) record_decode_error(p, TSQ_ERR_CORRUPT_BLOB);
+    __syncthreads();
+  }
+
+  // ---- the row leaves in one bulk store ----
+  if (tid == 0) {
+    fence_proxy_async_smem();
+    bulk_s2g(p.y + static_cast<size_t>(t) * p.hidden, smem_dyn, p.hidden * 2u);
+    bulk_commit();
+    bulk_wait_read_all();
+  }
+}
+
+}  // namespace
+
+size_t decode_smem_bytes(uint32_t row_bytes) { return (static_cast<size_t>(row_bytes) + 127u) & ~static_cast<size_t>(127u); }
+
+cudaError_t decode_kernel_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm) {
+  const void* fn = bf16 ? reinterpret_cast<const void*>(&decode_kernel<true>)
+                        : reinterpret_cast<const void*>(&decode_kernel<false>);
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads, smem);
+}
+
+cudaError_t launch_decode(const DecodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream) {
+  if (p.dtype == TSQ_BF16) {
+    decode_kernel<true><<<grid, threads, smem, stream>>>(p);
+  } else {
+    decode_kernel<false><<<grid, threads, smem, stream>>>(p);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace tsq

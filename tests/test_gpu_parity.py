@@ -1,0 +1,261 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tsq_ref as R
+from paper_2511_04002_b200 import binding as B
+from paper_2511_04002_b200 import synth
+from tests._parity import assert_blobs_equal, full_parity, gpu_decode, gpu_encode
+
+pytestmark = pytest.mark.gpu
+INF = float("inf")
+
+
+def rand16(shape, dtype, seed, scale=1.0, outlier_rate=0.0):
+    g = torch.Generator().manual_seed(seed)
+    v = torch.randn(shape, generator=g) * scale
+    if outlier_rate > 0:
+        hit = torch.rand(shape, generator=g) < outlier_rate
+        v = torch.where(hit, v * 40, v)
+    return v.to(dtype).contiguous()
+
+
+# ------------------------------------------------------------------ tiny and ragged shapes
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("shape", [(1, 8), (1, 32), (3, 40), (2, 4096), (5, 72), (7, 4104), (3, 264), (300, 8)])
+def test_small_shapes(dtype, shape):
+    x = rand16(shape, dtype, seed=shape[0] * 1000 + shape[1], scale=2.0, outlier_rate=0.02)
+    full_parity(x, 6.0, [2, 4, 8], 0.2)
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("delta", [-1.0, 0.0, 0.25, 0.5, 1.0, 1e9])
+@pytest.mark.parametrize("bits", [[2, 4, 8], [2, 3, 4, 8], [2, 3, 4, 5, 6, 7, 8], [8], [3], [2, 5]])
+def test_every_candidate_is_exercised(dtype, delta, bits):
+    T, H = 48, 1024
+    x = rand16((T, H), dtype, seed=len(bits) * 7 + int(delta * 4) % 5, scale=1.0, outlier_rate=0.001)
+    # rows whose bulk is small against their range drop to low levels
+    x[::3] = (x[::3].float().abs() ** 3 * 0.05).to(dtype) * torch.sign(x[::3].float()).to(dtype)
+    gpu_blob, _ = full_parity(x, 6.0, bits, delta)
+    chosen = set(R.sections(gpu_blob)["bits"].tolist())
+    if delta >= 1e9:
+        assert chosen == {bits[0]}
+    if delta < 0:
+        assert chosen == {bits[-1]}
+
+
+@pytest.mark.parametrize("hidden", [16384, 65536])
+def test_long_rows(hidden):
+    x = rand16((5, hidden), torch.bfloat16, seed=hidden, scale=1.5, outlier_rate=0.001)
+    full_parity(x, 6.0, [2, 4, 8], 0.2)
+
+
+# ------------------------------------------------------------------ adversarial rows
+
+def _special_rows(dtype, H=256):
+    rows = []
+    z = torch.zeros(H)
+    rows.append(z.clone())                                   # all zero
+    rows.append(torch.full((H,), 2.5))                       # constant
+    rows.append(torch.full((H,), -3.0))                      # constant negative
+    r = torch.randn(H); r[0] = 0.0; r[1] = -0.0; rows.append(r)
+    r = torch.randn(H) * 100; rows.append(r)                 # mostly outliers
+    r = torch.randn(H) * 0.01; rows.append(r)                # no outliers
+    r = torch.randn(H); r[3] = float("nan"); r[5] = INF; r[7] = -INF; rows.append(r)
+    r = torch.randn(H); r[10] = 6.0; r[11] = -6.0; r[12] = 5.99; rows.append(r)      # |x| == tau
+    r = (torch.arange(H) % 9).float() * 0.5; rows.append(r)  # many exact .5 ties in m / s
+    r = torch.arange(H).float() / H + 100.0; rows.append(r)  # narrow range far from zero -> large zero-point
+    r = torch.ones(H) * 4; r[0] = 4.004; rows.append(r)      # two adjacent values
+    r = torch.randn(H).abs() + 1.0; rows.append(r)           # non-zero minimum
+    x = torch.stack(rows).to(dtype)
+    # subnormal rows, built from raw patterns
+    sub = torch.zeros((2, H), dtype=dtype)
+    raw = synth.raw_u16(sub).copy()
+    rng = np.random.default_rng(1)
+    raw[0] = rng.integers(0, 0x0400 if dtype == torch.float16 else 0x0080, H).astype(np.uint16)
+    raw[1] = rng.integers(0, 0x0400 if dtype == torch.float16 else 0x0080, H).astype(np.uint16) | \
+        (rng.integers(0, 2, H).astype(np.uint16) << 15)
+    raw[1, ::5] = 0x3c00 if dtype == torch.float16 else 0x3f80   # subnormals next to 1.0
+    sub = synth.from_raw_u16(raw, "f16" if dtype == torch.float16 else "bf16")
+    return torch.cat([x, sub]).contiguous()
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("tau", [6.0, INF, 0.0, -1.0, 1e-7, 70000.0])
+def test_special_rows(dtype, tau):
+    full_parity(_special_rows(dtype), tau, [2, 4, 8], 0.2)
+    full_parity(_special_rows(dtype), tau, [2, 3, 4, 5, 6, 7, 8], 0.5)
+
+
+def test_huge_and_tiny_bf16_scales():
+    H = 512
+    g = torch.Generator().manual_seed(9)
+    big = (torch.randn((4, H), generator=g) * 1e37).to(torch.bfloat16)       # scale above 2^100
+    tiny = (torch.randn((4, H), generator=g) * 1e-36).to(torch.bfloat16)     # scale below 2^-100
+    x = torch.cat([big, tiny]).contiguous()
+    full_parity(x, INF, [2, 4, 8], 0.2)
+    full_parity(x, 1e30, [4, 8], 1.0)
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_all_16bit_magnitudes_appear(dtype):
+    # every finite non-negative pattern, shuffled into rows, so each rounding boundary meets a real value
+    top = 0x7c00 if dtype == torch.float16 else 0x7f80
+    pats = np.arange(top, dtype=np.uint32).astype(np.uint16)
+    rng = np.random.default_rng(0)
+    H = 1024
+    rows = []
+    for lo_exp in range(0, top, 2048):
+        seg = pats[lo_exp:lo_exp + 2048].copy()
+        rng.shuffle(seg)
+        rows.append(seg[:H]); rows.append(seg[H:2 * H] if seg.size >= 2 * H else np.resize(seg, H))
+    raw = np.stack(rows)
+    raw |= (rng.integers(0, 2, raw.shape).astype(np.uint16) << 15)
+    x = synth.from_raw_u16(raw, "f16" if dtype == torch.float16 else "bf16")
+    full_parity(x, INF, [2, 3, 4, 5, 6, 7, 8], 0.3)
+
+
+# ------------------------------------------------------------------ the paper-shaped workloads
+
+def test_c1_prefill():
+    w = synth.c1_prefill()
+    full_parity(synth.make(w), w.tau, w.bits, w.delta)
+
+
+def test_c2_decode_steps_share_one_workspace():
+    w = synth.c2_decode_steps(steps=12)
+    plan = B.Plan(torch.float16, w.recipe.hidden, w.recipe.tokens, w.tau, list(w.bits), w.delta)
+    blob, ws = plan.alloc()
+    for i in range(w.steps):
+        x = synth.make(w, i)
+        ref = R.encode(synth.raw_u16(x), R.F16, w.tau, list(w.bits), w.delta)
+        _, got, _ = gpu_encode(plan, x, ws=ws, blob=blob)
+        assert_blobs_equal(got, ref)
+        assert np.array_equal(gpu_decode(plan, blob, w.recipe.tokens, ws), R.decode(ref))
+    assert plan.workspace_status(ws) == (0, 0)
+
+
+def test_c3_13b_prefill():
+    w = synth.c3_13b_prefill()
+    full_parity(synth.make(w), w.tau, w.bits, w.delta, check_cross=False)
+
+
+def test_c4_70b_prefill_reduced():
+    w = synth.c4_70b_prefill(tokens=768)
+    full_parity(synth.make(w), w.tau, w.bits, w.delta, check_cross=False)
+
+
+@pytest.mark.parametrize("i_tok", [0, 1, 2])
+@pytest.mark.parametrize("i_rate", [0, 1, 2])
+@pytest.mark.parametrize("i_dtype", [0, 1])
+def test_c5_sweep_small(i_tok, i_rate, i_dtype):
+    w = synth.c5_sweep_point(i_tok, i_rate, i_dtype)
+    full_parity(synth.make(w), w.tau, w.bits, w.delta, check_cross=False)
+
+
+# ------------------------------------------------------------------ asynchronous conditions and errors
+
+def test_outlier_overflow_is_reported():
+    x = rand16((6, 512), torch.float16, seed=3, scale=3.0, outlier_rate=0.05)
+    gpu_blob, ref_blob = full_parity(x, 6.0, [2, 4, 8], 0.2, max_outliers=10)
+    assert R.header(gpu_blob)["status"] == 6
+    plan = B.Plan(torch.float16, 512, 6, 6.0, [2, 4, 8], 0.2, 10)
+    blob, _, ws = gpu_encode(plan, x)
+    assert plan.workspace_status(ws)[0] == 6
+    y = gpu_decode(plan, blob, 6, ws, fill=1.0)              # decoder refuses the blob, writes nothing
+    assert np.all(y == synth.raw_u16(torch.ones(1, dtype=torch.float16))[0])
+    assert plan.workspace_status(ws)[1] == 6
+    plan.workspace_init(ws)
+    x2 = rand16((6, 512), torch.float16, seed=4, scale=0.5)
+    _, got, _ = gpu_encode(plan, x2, ws=ws, blob=blob)       # the same buffers work again
+    assert_blobs_equal(got, R.encode(synth.raw_u16(x2), R.F16, 6.0, [2, 4, 8], 0.2, 10))
+
+
+def test_decoder_rejects_corrupt_blobs_without_writing():
+    x = rand16((4, 256), torch.float16, seed=5, scale=1.0, outlier_rate=0.01)
+    plan = B.Plan(torch.float16, 256, 4, 6.0, [2, 4, 8], 0.2)
+    blob, host, ws = gpu_encode(plan, x)
+    one = synth.raw_u16(torch.ones(1, dtype=torch.float16))[0]
+    lay = R.layout(256, 4, 8, 0)
+    cases = []
+    b = host.copy(); b[0] ^= 0xff; cases.append(b)                                 # magic
+    b = host.copy(); b[16] = 3; cases.append(b)                                    # tokens in header
+    b = host.copy(); b[lay["bits"] + 1] = 9; cases.append(b)                       # bit-width out of range
+    b = host.copy(); b[lay["word_off"] + 4:lay["word_off"] + 8] = 255; cases.append(b)   # offset out of range
+    b = host.copy(); b[lay["out_ptr"] + 8:lay["out_ptr"] + 12] = 255; cases.append(b)    # CSR pointer out of range
+    for bad in cases:
+        plan.workspace_init(ws)
+        y = gpu_decode(plan, torch.from_numpy(bad).cuda(), 4, ws, fill=1.0)
+        assert plan.workspace_status(ws)[1] == 5
+        changed_rows = np.nonzero((y != one).any(axis=1))[0]
+        assert changed_rows.size < 4                          # the offending rows (or all of them) are untouched
+    plan.workspace_init(ws)
+    y = gpu_decode(plan, blob, 4, ws)
+    assert plan.workspace_status(ws) == (0, 0)
+    assert np.array_equal(y, R.decode(host))
+
+
+def test_argument_errors_are_synchronous():
+    plan = B.Plan(torch.float16, 256, 4, 6.0, [2, 4, 8], 0.2)
+    blob, ws = plan.alloc()
+    x = torch.zeros((4, 256), dtype=torch.float16, device="cuda")
+    with pytest.raises(B.TsqError) as e:
+        plan.encode(x, blob[:128], ws)
+    assert e.value.status == 3
+    with pytest.raises(B.TsqError) as e:
+        plan.encode(x, blob, ws[:32])
+    assert e.value.status == 3
+    with pytest.raises(B.TsqError) as e:
+        plan.encode(torch.zeros((5, 256), dtype=torch.float16, device="cuda"), blob, ws)
+    assert e.value.status == 1
+    with pytest.raises(B.TsqError) as e:
+        plan.encode(x, blob[8:], ws)                          # misaligned blob
+    assert e.value.status == 1
+    for bad in ([], [1, 4], [4, 4], [2, 9]):
+        with pytest.raises(B.TsqError):
+            B.Plan(torch.float16, 256, 4, 6.0, bad)
+    with pytest.raises(B.TsqError) as e:
+        B.Plan(torch.float16, 100, 4, 6.0, [2, 4])
+    assert e.value.status == 2
+
+
+def test_empty_call_writes_a_valid_blob():
+    plan = B.Plan(torch.bfloat16, 512, 16, 6.0, [2, 4, 8], 0.2)
+    blob, ws = plan.alloc(0)
+    x = torch.zeros((0, 512), dtype=torch.bfloat16, device="cuda")
+    plan.encode(x, blob, ws)
+    torch.cuda.synchronize()
+    ref = R.encode(np.zeros((0, 512), np.uint16), R.BF16, 6.0, [2, 4, 8], 0.2)
+    assert np.array_equal(blob.cpu().numpy()[:64], ref[:64])
+    y = torch.zeros((0, 512), dtype=torch.bfloat16, device="cuda")
+    plan.decode(blob, 0, y, ws)
+    # the plan still serves a non-empty call afterwards, with the same workspace size
+    blob2, ws2 = plan.alloc(16)
+    xs = rand16((16, 512), torch.bfloat16, seed=8)
+    _, got, _ = gpu_encode(plan, xs, ws=ws2, blob=blob2)
+    assert_blobs_equal(got, R.encode(synth.raw_u16(xs), R.BF16, 6.0, [2, 4, 8], 0.2))
+
+
+def test_run_to_run_determinism_and_host_calls():
+    w = synth.c5_sweep_point(2, 2, 1)
+    x = synth.make(w)
+    plan = B.Plan(x.dtype, w.recipe.hidden, w.recipe.tokens, w.tau, list(w.bits), w.delta)
+    blob, ws = plan.alloc()
+    _, a, _ = gpu_encode(plan, x, ws=ws, blob=blob)
+    blob.zero_()
+    _, b, _ = gpu_encode(plan, x, ws=ws, blob=blob)
+    assert_blobs_equal(a, b)
+    # host-buffer entry points: same bytes as the device calls
+    T = w.recipe.tokens
+    x_pin = x.pin_memory()
+    blob_host = torch.zeros(blob.numel(), dtype=torch.uint8).pin_memory()
+    x_dev = torch.empty_like(x, device="cuda")
+    payload = plan.encode_host(x_pin, blob_host, x_dev, blob, ws)
+    assert payload == plan.blob_info(blob).payload_bytes
+    assert_blobs_equal(blob_host.numpy(), a)
+    y_host = torch.empty_like(x).pin_memory()
+    y_dev = torch.empty_like(x, device="cuda")
+    plan.decode_host(blob_host, T, y_host, blob, y_dev, ws)
+    assert np.array_equal(synth.raw_u16(y_host), R.decode(a))
