@@ -1,0 +1,462 @@
+#!/usr/bin/env python
+"""Throughput of the TS + TAB-Q codec on B200: one "step" = tsq_encode followed by tsq_decode of one
+[tokens x hidden] hidden state (threshold splitting, Eq. "ts"; token-wise TAB-Q, Algorithm 1;
+restore, Eq. "dequnt"), through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl tsq|reference] [--workload NAME]
+
+Prints ONE JSON line.  `value` is algorithmic GB/s (bytes the method must move: the 16-bit tensor in,
+the payload out, and the mirror for decode) with every buffer resident in HBM; `e2e` is the same
+figure through the host-buffer entry points with the host<->device copies inside the timed region;
+`roofline` is the slower of the two kernels against the measured HBM copy rate; `cpu_baseline` is the
+single-threaded CPU oracle on the same tensor; `decode_step` is the per-call latency of the
+decode-step workload (512 independent 64 x 4096 tensors).
+
+With N > 1 (one process per GPU, launched by torch.distributed.run) every rank encodes and decodes
+its own tensor: tokens are independent, there is no exchange step, so the job scales weakly with no
+collective on the data path.  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2511_04002_b200 import synth
+
+METRIC = "TS+TAB-Q encode+decode throughput (algorithmic bytes: 16-bit tensor + payload, both directions)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
+# under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
+# (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
+NCU_TRAFFIC = {
+    # "encode": {"sha256": "...", "bytes_per_token": ..., "hidden": 8192, "dtype": "bf16"},
+}
+
+
+def workload_by_name(name: str, tokens: int | None):
+    if name == "c4":
+        return synth.c4_70b_prefill(tokens or 8192)
+    if name == "c3":
+        w = synth.c3_13b_prefill()
+    elif name == "c1":
+        w = synth.c1_prefill()
+    elif name.startswith("c5"):
+        # c5:<i_tok>:<i_rate>:<i_dtype>
+        parts = [int(v) for v in name.split(":")[1:]] or [4, 1, 0]
+        w = synth.c5_sweep_point(*parts)
+    else:
+        raise SystemExit("unknown workload %r" % name)
+    if tokens:
+        from dataclasses import replace
+        w = replace(w, recipe=replace(w.recipe, tokens=tokens), name=w.name + "_tokens%d" % tokens)
+    return w
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ---------------------------------------------------------------------------------------------------
+# clocks: sampled on a thread during the timed region (read-only NVML queries)
+
+_REASONS = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+            0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+            0x100: "display_clock_setting"}
+
+
+class ClockSampler:
+    def __init__(self, device_index: int, period_s: float = 0.004):
+        self.period = period_s
+        self.samples, self.reason_bits = [], 0
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            uuid = torch.cuda.get_device_properties(device_index).uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-%s" % uuid).encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _poll(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": [n for b, n in _REASONS.items() if self.reason_bits & b], "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------------------------
+# the CPU oracle legs (the only places this file touches oracle/)
+
+def oracle_pass(raw: np.ndarray, w) -> tuple[float, int]:
+    """One encode + decode of `raw` by the CPU oracle. Returns (seconds, payload bytes)."""
+    from oracle import tsq_ref as R
+    code = R.F16 if w.recipe.dtype == "f16" else R.BF16
+    t0 = time.perf_counter()
+    blob = R.encode(raw, code, w.tau, list(w.bits), w.delta)
+    y = R.decode(blob)
+    dt = time.perf_counter() - t0
+    h = R.header(blob)
+    T = raw.shape[0]
+    payload = 64 + 9 * T + 8 * (T + 1) + 4 * h["total_words"] + 4 * h["total_outliers"]
+    assert y.shape == raw.shape
+    return dt, payload
+
+
+def step_bytes(tokens: int, hidden: int, payload: int) -> int:
+    """Algorithmic bytes of one encode + decode: tensor in, payload out; payload in, tensor out."""
+    return 2 * (tokens * hidden * 2 + payload)
+
+
+def cpu_baseline(x_cpu: torch.Tensor, w, budget_s: float = 12.0):
+    raw = synth.raw_u16(x_cpu)
+    T, H = raw.shape
+    oracle_pass(raw[: min(T, 8)], w)                      # builds and loads the oracle, warms the caches
+    elapsed, passes, payload = 0.0, 0, 0
+    while elapsed < budget_s and passes < 50:
+        dt, payload = oracle_pass(raw, w)
+        elapsed += dt
+        passes += 1
+    gbs = passes * step_bytes(T, H, payload) / elapsed / 1e9
+    return {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "%d full pass(es) of the %dx%d tensor (encode + decode), single thread, %.1f s" % (
+                passes, T, H, elapsed)}
+
+
+def run_reference(args, w):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    x = synth.make(w)
+    raw = synth.raw_u16(x)
+    T, H = raw.shape
+    dt, _ = oracle_pass(raw[: min(T, 16)], w)
+    dt, _ = oracle_pass(raw[: min(T, 16)], w)
+    per_token = dt / min(T, 16)
+    S = int(max(1, min(T, 60.0 / (per_token * (args.steps + args.warmup)))))
+    sample = raw[:S]
+    for _ in range(args.warmup):
+        oracle_pass(sample, w)
+    total, payload = 0.0, 0
+    for _ in range(args.steps):
+        dt, payload = oracle_pass(sample, w)
+        total += dt
+    gbs = args.steps * step_bytes(S, H, payload) / total / 1e9
+    sample_txt = "first %d of %d tokens per step, single thread" % (S, T)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "tokens": T, "hidden": H, "tau": w.tau, "bits": list(w.bits), "delta": w.delta,
+                   "seed": w.seed, "sample": sample_txt},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample_txt},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------
+# the CUDA arm
+
+class BufferSet:
+    def __init__(self, plan, x_cpu: torch.Tensor):
+        self.x = x_cpu.cuda(non_blocking=False)
+        self.blob, self.ws = plan.alloc(x_cpu.shape[0])
+        self.y = torch.empty_like(self.x)
+
+
+def decode_step_latency(B, device, n_calls: int):
+    """Per-call latency on the decode-step workload: independent [64 x 4096] fp16 tensors, each with its
+    own input, blob and output resident on the device; calls issued back to back on one stream, and
+    the same train replayed from a CUDA graph (no host launch cost)."""
+    w = synth.c2_decode_steps(n_calls)
+    T, H = w.recipe.tokens, w.recipe.hidden
+    plan = B.Plan(torch.float16, H, T, w.tau, list(w.bits), w.delta, device=device)
+    blob_bytes, ws_bytes = plan.sizes(T)
+    xs = torch.empty((n_calls, T, H), dtype=torch.float16, device="cuda")
+    for i in range(n_calls):
+        xs[i].copy_(synth.make(w, i))
+    blobs = torch.empty((n_calls, (blob_bytes + 255) // 256 * 256), dtype=torch.uint8, device="cuda")
+    ys = torch.empty_like(xs)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    plan.workspace_init(ws)
+    stream = torch.cuda.Stream()
+    out = {"workload": w.name, "calls": n_calls}
+
+    xl, bl, yl = list(xs.unbind(0)), list(blobs.unbind(0)), list(ys.unbind(0))
+
+    def enc_train():
+        for i in range(n_calls):
+            plan.encode(xl[i], bl[i], ws, stream)
+
+    def dec_train():
+        for i in range(n_calls):
+            plan.decode(bl[i], T, yl[i], ws, stream)
+
+    def pair_train():
+        for i in range(n_calls):
+            plan.encode(xl[i], bl[i], ws, stream)
+            plan.decode(bl[i], T, yl[i], ws, stream)
+
+    def timed(fn, reps=3):
+        best = float("inf")
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            stream.synchronize()
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            stream.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return 1e3 * best / n_calls
+
+    with torch.cuda.stream(stream):
+        enc_train(); dec_train()                                           # warm-up
+        stream.synchronize()
+        out["stream_us_per_call"] = {"encode": timed(enc_train), "decode": timed(dec_train),
+                                     "encode+decode": timed(pair_train)}
+        graphs = {}
+        for name, fn in (("encode", enc_train), ("decode", dec_train), ("encode+decode", pair_train)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+            graphs[name] = g
+        out["graph_us_per_call"] = {k: timed(g.replay) for k, g in graphs.items()}
+    info = plan.blob_info(bl[0])
+    assert info.status == 0 and plan.workspace_status(ws) == (0, 0)
+    out["payload_bytes_call0"] = info.payload_bytes
+    return out
+
+
+def run_tsq(args, w):
+    from paper_2511_04002_b200 import binding as B
+    B.lib()                                                # raises if the CUDA library is missing
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the tsq library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    T, H = w.recipe.tokens, w.recipe.hidden
+    dt = synth.torch_dtype(w.recipe.dtype)
+    plan = B.Plan(dt, H, T, w.tau, list(w.bits), w.delta, device=local)
+
+    # distinct tensors rotate through the timed loop so that no step finds its input in L2
+    n_sets = max(1, args.sets)
+    x0 = synth.generate(w.recipe, w.seed + 100000 * rank)
+    sets = [BufferSet(plan, x0)]
+    for k in range(1, n_sets):
+        sets.append(BufferSet(plan, synth.generate(w.recipe, w.seed + 100000 * rank + 1000 * k)))
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        s = sets[i % n_sets]
+        plan.encode(s.x, s.blob, s.ws)
+        plan.decode(s.blob, T, s.y, s.ws)
+    torch.cuda.synchronize()
+    infos = [plan.blob_info(s.blob) for s in sets]
+    for s, info in zip(sets, infos):
+        assert info.status == 0 and plan.workspace_status(s.ws) == (0, 0), "codec reported an error"
+    payloads = [i.payload_bytes for i in infos]
+    x_bytes = T * H * 2
+
+    K = args.steps
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K + 1)]
+    launches0 = B.kernel_launch_count()
+    barrier()
+    with ClockSampler(local) as clocks:
+        ev[0].record(stream)
+        for i in range(K):
+            s = sets[i % n_sets]
+            plan.encode(s.x, s.blob, s.ws)
+            ev[2 * i + 1].record(stream)
+            plan.decode(s.blob, T, s.y, s.ws)
+            ev[2 * i + 2].record(stream)
+        torch.cuda.synchronize()
+    barrier()
+    launches = B.kernel_launch_count() - launches0
+    total_ms = ev[0].elapsed_time(ev[2 * K])
+    enc_ms = sum(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(K)) / K
+    dec_ms = sum(ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(K)) / K
+    bytes_done = sum(2 * (x_bytes + payloads[i % n_sets]) for i in range(K))
+    for s in sets:
+        assert plan.workspace_status(s.ws) == (0, 0), "codec reported an error in the timed region"
+
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        b = torch.tensor([float(bytes_done), float(launches)], dtype=torch.float64, device="cuda")
+        dist.all_reduce(b, op=dist.ReduceOp.SUM)
+        bytes_done, launches = float(b[0].item()), int(b[1].item())
+
+    # ---- end to end: host tensors in and out, copies inside the timed region (every rank, in parallel)
+    e2e = None
+    if not args.no_e2e:
+        s = sets[0]
+        x_pin = x0.pin_memory()
+        blob_pin = torch.empty(s.blob.numel(), dtype=torch.uint8).pin_memory()
+        y_pin = torch.empty_like(x0).pin_memory()
+        n_e2e = max(3, min(K, args.e2e_steps))
+        for _ in range(2):
+            payload = plan.encode_host(x_pin, blob_pin, s.x, s.blob, s.ws)
+            plan.decode_host(blob_pin, T, y_pin, s.blob, s.y, s.ws)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n_e2e):
+            payload = plan.encode_host(x_pin, blob_pin, s.x, s.blob, s.ws)
+            plan.decode_host(blob_pin, T, y_pin, s.blob, s.y, s.ws)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * n_e2e * 2 * (x_bytes + payload) / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": x_bytes + payload, "d2h_bytes_per_step": payload + x_bytes,
+               "steps": n_e2e, "ms_per_step": e2e_ms / n_e2e,
+               "api": "tsq_encode_host + tsq_decode_host, pinned host buffers"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak_gbs()
+    p0 = payloads[0]
+    kern = {
+        "encode": {"ms": enc_ms, "bytes": x_bytes + p0, "GB/s": (x_bytes + p0) / (enc_ms * 1e-3) / 1e9},
+        "decode": {"ms": dec_ms, "bytes": x_bytes + p0, "GB/s": (x_bytes + p0) / (dec_ms * 1e-3) / 1e9},
+    }
+    dom = "encode" if enc_ms >= dec_ms else "decode"
+    traffic = None
+    rec = NCU_TRAFFIC.get(dom)
+    if rec:
+        src = os.path.join(ROOT, "paper_2511_04002_b200", "csrc", "tsq_%s.cu" % dom)
+        with open(src, "rb") as f:
+            same = hashlib.sha256(f.read()).hexdigest() == rec["sha256"]
+        if same and rec["hidden"] == H and rec["dtype"] == w.recipe.dtype:
+            traffic = rec["bytes_per_token"] * T
+    roofline = {"bound": "hbm", "kernel": "tsq %s_kernel" % dom, "achieved": kern[dom]["GB/s"], "peak": peak,
+                "unit": "GB/s", "frac": kern[dom]["GB/s"] / peak, "traffic": traffic, "peak_source": peak_kind,
+                "bytes_per_launch": kern[dom]["bytes"], "ms_per_launch": kern[dom]["ms"],
+                "frac_of_nominal_8TBs": kern[dom]["GB/s"] / 8000.0}
+    for k in kern.values():
+        k["frac"] = k["GB/s"] / peak
+
+    line = {
+        "metric": METRIC, "value": bytes_done / (total_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": args.warmup, "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "tokens": T, "hidden": H, "elem": w.recipe.dtype, "tau": w.tau,
+                   "bits": list(w.bits), "delta": w.delta, "seed": w.seed, "tokens_per_gpu": T,
+                   "parallelism": "token ranges per GPU, no collective",
+                   "l2": "rotating %d distinct input/blob/output sets (%.0f MB touched between reuses)" % (
+                       n_sets, n_sets * (2 * x_bytes + p0) / 1e6),
+                   "payload_bytes": p0, "compression_ratio": x_bytes / p0},
+        "clocks": clocks.summary(), "gpu_launches": launches, "kernels": kern, "roofline": roofline,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(x0, w)
+    if world == 1 and not args.no_decode_step:
+        for s in sets[1:]:
+            del s.x, s.blob, s.y
+        line["decode_step"] = decode_step_latency(B, local, args.decode_calls)
+    if world > 1:
+        dist.destroy_process_group()
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="tsq", choices=["tsq", "reference"])
+    ap.add_argument("--workload", default="c4", help="c4 (default, the 8192x8192 bf16 prefill), c3, c1, c5:<tok>:<rate>:<dtype>")
+    ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (small profiling cases)")
+    ap.add_argument("--sets", type=int, default=3, help="distinct buffer sets rotated through the timed loop")
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--decode-calls", type=int, default=512)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode-step", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    w = workload_by_name(args.workload, args.tokens or None)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_tsq(args, w)
+
+
+if __name__ == "__main__":
+    main()
