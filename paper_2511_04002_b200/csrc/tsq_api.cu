@@ -62,10 +62,11 @@ struct tsq_plan {
   int32_t bmax;
   int32_t s_max;
   uint32_t thr16;
-  int threads;
-  uint32_t stages;
-  size_t enc_smem, dec_smem;
-  int enc_grid_limit;  // CTAs that are co-resident on the device
+  int threads;                      // decoder CTA size
+  uint32_t enc_row_stride, enc_warp_stride;
+  int enc_warps;                    // warps per encoder CTA that fit in shared memory
+  int sms;
+  size_t dec_smem;
   size_t workspace_bytes;
 };
 
@@ -127,15 +128,12 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   p->thr16 = threshold_pattern(dtype, tau);
   p->threads = static_cast<int>(((p->units + 31u) / 32u) * 32u);
   if (p->threads > kMaxThreads) p->threads = kMaxThreads;
-  const size_t row_stride = (static_cast<size_t>(p->row_bytes) + 127u) & ~static_cast<size_t>(127u);
-  size_t stages = (54u * 1024u) / row_stride;
-  if (stages < 1) stages = 1;
-  if (stages > static_cast<size_t>(kMaxStages)) stages = kMaxStages;
-  p->stages = static_cast<uint32_t>(stages);
-  p->enc_smem = encode_smem_bytes(p->units, p->row_bytes, p->stages);
+  // encoder shared memory per warp: the row (128-byte aligned) and the list of units holding outliers
+  p->enc_row_stride = (p->row_bytes + 127u) & ~127u;
+  p->enc_warp_stride = p->enc_row_stride + ((p->units * 2u + 127u) & ~127u);
   p->dec_smem = decode_smem_bytes(p->row_bytes);
   const unsigned long long desc = T > 0 ? T : 1;
-  p->workspace_bytes = sizeof(WsControl) + 2 * sizeof(unsigned long long) * desc;
+  p->workspace_bytes = static_cast<size_t>(align16(sizeof(WsControl) + 12ull * desc));
 
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) {
@@ -145,17 +143,25 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   int prev_dev = 0;
   cudaGetDevice(&prev_dev);
   bool ok = cudaSetDevice(device) == cudaSuccess;
-  int sms = 0, enc_blocks = 0, dec_blocks = 0;
+  int sms = 0, dec_blocks = 0, smem_optin = 0;
   ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess;
-  ok = ok && encode_kernel_attrs(dtype == TSQ_BF16, p->threads, p->enc_smem, &enc_blocks) == cudaSuccess;
+  ok = ok && cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) == cudaSuccess;
+  if (ok) {
+    // one encoder CTA per SM, as many row slots as fit beside the kernel's static shared memory
+    long long w = (static_cast<long long>(smem_optin) - 1024) / static_cast<long long>(p->enc_warp_stride);
+    if (w > kEncMaxWarps) w = kEncMaxWarps;
+    p->enc_warps = static_cast<int>(w);
+    ok = w >= 1;
+  }
+  ok = ok && encode_kernel_attrs(dtype == TSQ_BF16, static_cast<size_t>(p->enc_warps) * p->enc_warp_stride) == cudaSuccess;
   ok = ok && decode_kernel_attrs(dtype == TSQ_BF16, p->threads, p->dec_smem, &dec_blocks) == cudaSuccess;
   cudaSetDevice(prev_dev);
-  if (!ok || enc_blocks < 1 || dec_blocks < 1 || sms < 1) {
+  if (!ok || dec_blocks < 1 || sms < 1) {
     cudaGetLastError();
     delete p;
     return TSQ_ERR_CUDA;
   }
-  p->enc_grid_limit = enc_blocks * sms;
+  p->sms = sms;
   *out = p;
   return TSQ_OK;
 }
@@ -181,7 +187,7 @@ tsq_status_t tsq_workspace_init(const tsq_plan_t* plan, void* ws_dev, size_t ws_
   if (ws_bytes < plan->workspace_bytes) return TSQ_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(ws_dev, 0, plan->workspace_bytes, st) != cudaSuccess) return TSQ_ERR_CUDA;
-  const uint32_t cap = static_cast<uint32_t>((plan->workspace_bytes - sizeof(WsControl)) / (2 * sizeof(unsigned long long)));
+  const uint32_t cap = static_cast<uint32_t>(plan->max_tokens > 0 ? plan->max_tokens : 1);
   workspace_init_kernel<<<1, 1, 0, st>>>(static_cast<WsControl*>(ws_dev), cap);
   g_launches.fetch_add(1);
   return cudaGetLastError() == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
@@ -202,8 +208,8 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
   p.blob = static_cast<unsigned char*>(blob_dev);
   p.ws = static_cast<WsControl*>(ws_dev);
   const unsigned long long desc = plan->max_tokens > 0 ? plan->max_tokens : 1;
-  p.desc_words = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(ws_dev) + sizeof(WsControl));
-  p.desc_outl = p.desc_words + desc;
+  p.desc = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(ws_dev) + sizeof(WsControl));
+  p.prefix_outl = reinterpret_cast<uint32_t*>(p.desc + desc);
   p.lay = L;
   p.tokens = static_cast<uint32_t>(tokens);
   p.hidden = plan->hidden;
@@ -213,15 +219,22 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
   p.n_bits = plan->n_bits;
   for (int i = 0; i < 8; ++i) p.bits[i] = plan->bits[i];
   p.s_max = plan->s_max;
-  p.stages = plan->stages;
   p.row_bytes = plan->row_bytes;
+  p.row_stride = plan->enc_row_stride;
+  p.warp_stride = plan->enc_warp_stride;
   p.dtype = static_cast<uint32_t>(plan->dtype);
   p.tau = plan->tau;
   p.delta = plan->delta;
 
-  int grid = tokens < plan->enc_grid_limit ? static_cast<int>(tokens) : plan->enc_grid_limit;
+  // rows are spread over the SMs first, then over the warps of each CTA
+  int grid = tokens < plan->sms ? static_cast<int>(tokens) : plan->sms;
   if (grid < 1) grid = 1;
-  const cudaError_t e = launch_encode(p, grid, plan->threads, plan->enc_smem, static_cast<cudaStream_t>(cuda_stream));
+  long long active = (tokens + grid - 1) / grid;
+  if (active > plan->enc_warps) active = plan->enc_warps;
+  if (active < 1) active = 1;
+  p.active_warps = static_cast<uint32_t>(active);
+  const cudaError_t e = launch_encode(p, grid, plan->enc_warps * 32, static_cast<size_t>(plan->enc_warps) * plan->enc_warp_stride,
+                                      static_cast<cudaStream_t>(cuda_stream));
   g_launches.fetch_add(1);
   return e == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
 }

@@ -13,8 +13,8 @@ namespace tsq {
 constexpr uint32_t kMagic = 0x31515354u;  // 'T','S','Q','1'
 constexpr uint32_t kVersion = 1u;
 constexpr int kMaxCand = 7;
-constexpr int kMaxThreads = 256;          // threads per CTA, one 32-element unit per thread per pass
-constexpr int kMaxStages = 4;             // rows in flight per CTA (bulk-copy ring)
+constexpr int kMaxThreads = 256;          // decoder: threads per CTA, one 32-element unit per thread per pass
+constexpr int kEncMaxWarps = 16;          // encoder: warps per CTA, one row in flight per warp
 
 struct BlobHeader {
   uint32_t magic, version, dtype, hidden, tokens, n_bits;
@@ -53,10 +53,9 @@ __host__ __device__ inline BlobLayout make_layout(uint32_t hidden, unsigned long
   return L;
 }
 
-// Workspace: a 64-byte control block followed by two arrays of 64-bit tile descriptors
-// (running totals of plane words and of outliers).  A descriptor is (tag << 32) | value with
-// tag = generation * 4 + flag; stale generations read as "not yet published", so the arrays
-// never need clearing between calls.
+// Workspace: a 64-byte control block, one 64-bit descriptor per token and one 32-bit outlier
+// prefix per token.  A descriptor is (tag << 32) | value with tag = generation * 4 + flag; stale
+// generations read as "not yet published", so the arrays never need clearing between calls.
 struct WsControl {
   uint32_t gen;          // generation of the last finished encode
   uint32_t ticket;       // next tile to hand out (self-resetting)
@@ -76,15 +75,17 @@ struct EncodeParams {
   const uint16_t* x;
   unsigned char* blob;
   WsControl* ws;
-  unsigned long long* desc_words;
-  unsigned long long* desc_outl;
+  unsigned long long* desc;                  // [max_tokens] tile descriptors
+  uint32_t* prefix_outl;                     // [max_tokens] inclusive outlier prefixes
   BlobLayout lay;
   uint32_t tokens, hidden, units, chunks;   // units = ceil(H/32), chunks = H/8
   uint32_t thr16;                            // smallest non-negative 16-bit pattern with value >= tau
   int32_t n_bits;
   int32_t bits[8];
   int32_t s_max;                             // floor(delta * H), clamped to [-1, INT32_MAX]
-  uint32_t stages, row_bytes;
+  uint32_t row_bytes;                        // bytes of one input row
+  uint32_t row_stride, warp_stride;          // shared memory: row slot, and row slot + unit list, per warp
+  uint32_t active_warps;                     // warps of each CTA that take rows
   uint32_t dtype;
   float tau, delta;
 };
@@ -101,9 +102,8 @@ struct DecodeParams {
 
 cudaError_t launch_encode(const EncodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
-cudaError_t encode_kernel_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm);
+cudaError_t encode_kernel_attrs(bool bf16, size_t smem);
 cudaError_t decode_kernel_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm);
-size_t encode_smem_bytes(uint32_t units, uint32_t row_bytes, uint32_t stages);
 size_t decode_smem_bytes(uint32_t row_bytes);
 
 }  // namespace tsq
