@@ -73,9 +73,10 @@ typedef struct {
  *   zp       i32 [tokens]      AIQ zero-point, restore = (code + zp) * s
  *   word_off u32 [tokens+1]    exclusive prefix sum of b* x WPP
  *   out_ptr  u32 [tokens+1]    CSR row pointers (exclusive prefix sum of per-token outlier counts)
- *   words    u32 [tokens x bmax x WPP]  token t owns b* planes of WPP words from word_off[t]:
+ *   words    u32 [tokens x bmax x WPP]  token t owns b* x WPP words from word_off[t], interleaved
+ *                  per group of 32 elements: word g*b* + k is plane k of elements 32g .. 32g+31,
  *                  plane 0 = sign bits of the inliers, plane 1+k = bit k of the magnitude codes;
- *                  bit i of word w belongs to element 32*w + i; pad bits are 0
+ *                  bit i of a group's word belongs to element 32g + i; pad bits are 0
  *   outl     u32 [outlier_capacity]     (column << 16) | original 16-bit pattern, columns ascending
  */
 

@@ -174,7 +174,8 @@ uint16_t float_to_raw16_nonneg(int dtype, float f) {
 // ---- blob layout ---------------------------------------------------------------------
 // header (64 B) | bits[T] u8 | scale[T] f32 | zp[T] i32 | word_off[T+1] u32 |
 // out_ptr[T+1] u32 | words[T*bmax*WPP] u32 | outl[capacity] u32 ; every section starts
-// on a 16-byte boundary.
+// on a 16-byte boundary.  Inside a token's b*WPP words the planes are interleaved per group of
+// 32 elements: word g*b + k is plane k of elements 32g .. 32g+31.
 
 struct Header {
   uint32_t magic, version, dtype, hidden, tokens, n_bits;
@@ -392,15 +393,16 @@ int tsq_ref_encode(int dtype, int hidden, long long tokens, float tau, const int
     o_bits[t] = (uint8_t)r.b;
     o_scale[t] = r.s;
     o_zp[t] = r.zp;
-    // bit-planes: plane 0 = sign, plane 1+k = bit k of the magnitude code; bit i of word w
-    // belongs to element 32*w + i; pad bits stay 0.
+    // bit-planes: plane 0 = sign, plane 1+k = bit k of the magnitude code.  Group g holds
+    // elements 32g .. 32g+31 and owns words g*b .. g*b + b-1 (one word per plane); bit i of a
+    // group's word belongs to element 32g + i; pad bits stay 0.
     uint32_t* wrow = o_words + word_off;
     for (int64_t j = 0; j < H; ++j) {
-      const uint64_t w = (uint64_t)j >> 5;
+      const uint64_t g = (uint64_t)j >> 5;
       const uint32_t bit = 1u << (j & 31);
-      if (sg[j]) wrow[w] |= bit;
+      if (sg[j]) wrow[g * r.b] |= bit;
       for (int k = 0; k < r.b - 1; ++k) {
-        if ((qbest[j] >> k) & 1) wrow[(uint64_t)(1 + k) * L.wpp + w] |= bit;
+        if ((qbest[j] >> k) & 1) wrow[g * r.b + 1 + k] |= bit;
       }
     }
     word_off += (uint64_t)r.b * L.wpp;
@@ -467,11 +469,11 @@ int tsq_ref_decode(const uint8_t* blob, unsigned long long blob_bytes, uint16_t*
     const uint32_t* wrow = i_words + wo;
     uint16_t* yrow = y + t * H;
     for (int64_t j = 0; j < H; ++j) {
-      const uint64_t w = (uint64_t)j >> 5;
+      const uint64_t g = (uint64_t)j >> 5;
       const int sh = (int)(j & 31);
       int32_t q = 0;
-      for (int k = 0; k < b - 1; ++k) q |= (int32_t)((wrow[(uint64_t)(1 + k) * L.wpp + w] >> sh) & 1u) << k;
-      const uint32_t sign = (wrow[w] >> sh) & 1u;
+      for (int k = 0; k < b - 1; ++k) q |= (int32_t)((wrow[g * b + 1 + k] >> sh) & 1u) << k;
+      const uint32_t sign = (wrow[g * b] >> sh) & 1u;
       const float mag = (float)(q + zp) * s;              // (T^ - Z) .* S with Z = -zp (R1)
       const uint16_t hbits = float_to_raw16_nonneg(dtype, mag);  // R15
       yrow[j] = (uint16_t)(hbits | (sign << 15));

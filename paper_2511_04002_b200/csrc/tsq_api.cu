@@ -63,7 +63,7 @@ struct tsq_plan {
   int32_t s_max;
   uint32_t thr16;
   int threads;                      // decoder CTA size
-  uint32_t enc_row_stride, enc_warp_stride;
+  uint32_t enc_row_stride, enc_warp_stride, enc_stash_cap;
   int enc_warps;                    // warps per encoder CTA that fit in shared memory
   int sms;
   size_t dec_smem;
@@ -128,9 +128,11 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   p->thr16 = threshold_pattern(dtype, tau);
   p->threads = static_cast<int>(((p->units + 31u) / 32u) * 32u);
   if (p->threads > kMaxThreads) p->threads = kMaxThreads;
-  // encoder shared memory per warp: the row (128-byte aligned) and the list of units holding outliers
+  // encoder shared memory per warp: the row (128-byte aligned) and a stash of one outlier per
+  // 32 elements (rows with more take a slower path)
   p->enc_row_stride = (p->row_bytes + 127u) & ~127u;
-  p->enc_warp_stride = p->enc_row_stride + ((p->units * 2u + 127u) & ~127u);
+  p->enc_stash_cap = (p->units * 4u + 127u) / 128u * 32u;
+  p->enc_warp_stride = p->enc_row_stride + p->enc_stash_cap * 4u;
   p->dec_smem = decode_smem_bytes(p->row_bytes);
   const unsigned long long desc = T > 0 ? T : 1;
   p->workspace_bytes = static_cast<size_t>(align16(sizeof(WsControl) + 12ull * desc));
@@ -222,6 +224,8 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
   p.row_bytes = plan->row_bytes;
   p.row_stride = plan->enc_row_stride;
   p.warp_stride = plan->enc_warp_stride;
+  p.stash_cap = plan->enc_stash_cap;
+  p.bulk_store = (plan->units % 4u == 0u) ? 1u : 0u;
   p.dtype = static_cast<uint32_t>(plan->dtype);
   p.tau = plan->tau;
   p.delta = plan->delta;

@@ -32,12 +32,24 @@ __device__ __forceinline__ void restore_units(const DecodeParams& p, const uint3
   extern __shared__ __align__(128) unsigned char smem_dyn[];
   uint4* stage4 = reinterpret_cast<uint4*>(smem_dyn);
   const float neg_bias = DIRECT ? 0.0f : -__fmul_rn(kTwo23, s);
+  const bool vec = (reinterpret_cast<uintptr_t>(words) & 15u) == 0;  // 16-byte loads of a group's words
   const uint32_t int_bias = kTwo23Bits + static_cast<uint32_t>(zp);
   for (uint32_t u = threadIdx.x; u < p.units; u += blockDim.x) {
-    uint32_t r[8];
+    // group u owns words u * b .. u * b + b - 1, one per plane
+    uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const uint32_t* src = words + static_cast<size_t>(u) * b;
+    if (vec && b == 8u) {
+      const uint4 lo = __ldg(reinterpret_cast<const uint4*>(src)), hi = __ldg(reinterpret_cast<const uint4*>(src) + 1);
+      r[0] = lo.x; r[1] = lo.y; r[2] = lo.z; r[3] = lo.w;
+      r[4] = hi.x; r[5] = hi.y; r[6] = hi.z; r[7] = hi.w;
+    } else if (vec && b == 4u) {
+      const uint4 lo = __ldg(reinterpret_cast<const uint4*>(src));
+      r[0] = lo.x; r[1] = lo.y; r[2] = lo.z; r[3] = lo.w;
+    } else {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      r[k] = (static_cast<uint32_t>(k) < b) ? __ldg(words + static_cast<size_t>(k) * p.lay.wpp + u) : 0u;
+      for (int k = 0; k < 8; ++k) {
+        if (static_cast<uint32_t>(k) < b) r[k] = __ldg(src + k);
+      }
     }
     transpose8x32(r);  // r[i] byte c = (code << 1 | sign) of element 8c + i
     const uint32_t rot = (u >> 1) & 3u;

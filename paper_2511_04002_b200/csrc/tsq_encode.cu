@@ -4,17 +4,29 @@
 // One WARP works on one token row at a time, and no two warps ever synchronise with each other:
 // a warp takes the next row by an atomic ticket, fetches it into its own shared-memory slot with
 // one bulk asynchronous copy (completion on the warp's own mbarrier), runs every pass of the
-// method on that copy, and writes the row's part of the blob.  The input is therefore read from
-// HBM exactly once, and while one warp waits (for its copy, or for the placement of its output)
-// the other warps of the SM keep the issue slots busy.
+// method on that copy, and sends the row's planes to the blob with one bulk asynchronous store.
+// The input is therefore read from HBM exactly once, and while one warp waits (for its copy, or
+// for the placement of its output) the other warps of the SM keep the issue slots busy.
+//
+// Passes over the slot:
+//   A      threshold split: per-token min / max of the inlier magnitudes; every outlier is copied
+//          (column, original pattern) to the warp's stash in column order and its slot is set to +0,
+//          which is what T_below holds there, so the later passes need no mask;
+//   B      Algorithm 1: AIQ codes at the top level and at each lower candidate, distortion sums;
+//   C      codes at the chosen level -> bytes (code << 1 | sign) -> 8 x 32 bit transpose -> the
+//          group's b* plane words, written over the front of the slot itself (group g's words end
+//          before group g's input begins, and a warp reads 32 groups before it writes them);
+//   then the placement is looked up and slot and stash leave for the blob.
 //
 // Variable-length placement: where a token's planes and CSR entries start is an exclusive prefix
 // sum over all earlier tokens.  It is resolved with a decoupled look-back over per-token
 // descriptors in the workspace.  Tickets are handed out in row order, so a row only ever waits
-// for rows held by warps that are already running.  A look-back step reads 256 descriptors at
-// once (eight independent loads per lane): with well over a hundred rows finishing per
-// microsecond, a narrower window cannot reach the nearest published prefix within one memory
-// round trip.  Every wait is bounded and fails into a status word.
+// for rows held by warps that are already running.  A row publishes its own sizes right after
+// pass B and looks back only after pass C, so that the wait for slower predecessors overlaps its
+// own packing.  A look-back step reads 256 descriptors at once (eight independent loads per
+// lane): with well over a hundred rows finishing per microsecond, a narrower window cannot reach
+// the nearest published prefix within one memory round trip.  Every wait is bounded and fails
+// into a status word.
 //
 // Arithmetic contract: the codes equal  clamp(rint(m / s) - zp, 0, Qmax)  with the IEEE binary32
 // quotient m / s.  Three evaluations of it exist, chosen per row:
@@ -29,7 +41,8 @@
 //             (the classical FMA division step, exact when r is the correctly rounded reciprocal
 //             and nothing over- or underflows), then the same 1.5 * 2^23 rounding.
 //   kDivide   the division instruction itself, for rows whose scale is so large or so small that
-//             the intermediate products of the other two could leave the normal range.
+//             the intermediate products of the other two could leave the normal range, or whose
+//             zero-point does not fit the packed 16-bit integer steps of the other two.
 
 #include "tsq_device.cuh"
 #include "tsq_internal.h"
@@ -38,19 +51,19 @@ namespace tsq {
 namespace {
 
 constexpr float kRoundMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer, ties to even
-constexpr int kRoundMagicBits = 0x4B400000;
 constexpr uint32_t kLookbackPollLimit = 1u << 20;
 constexpr uint32_t kCopyPollLimit = 1u << 20;
 constexpr int kLookbackDepth = 8;  // descriptors each lane reads per look-back step
 
 // AIQ parameters of one candidate level for one row (Eq. "Proposed").
 struct Level {
-  float s;    // scale
-  float r;    // fl(1 / s), fast path only
-  int zp;     // zero-point rint(m_min / s)
-  int bias;   // kRoundMagicBits + zp
-  int qmax;   // 2^(b-1) - 1
-  bool fast;  // scale in the range where the FMA paths are provably safe
+  float s;       // scale
+  float r;       // fl(1 / s)
+  int zp;        // zero-point rint(m_min / s)
+  int qmax;      // 2^(b-1) - 1
+  uint32_t nz2;  // -zp in both 16-bit halves
+  uint32_t qm2;  // qmax in both 16-bit halves
+  bool fast;     // scale and zero-point in the range where the FMA paths are provably safe
 };
 
 enum Mode : int { kFast = 0, kRefined = 1, kDivide = 2 };
@@ -61,25 +74,48 @@ __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
   const float range = __fsub_rn(mmax, mmin);
   c.s = range > 0.0f ? __fdiv_rn(range, static_cast<float>(c.qmax)) : (mmax > 0.0f ? mmax : 1.0f);
   c.zp = __float2int_rn(__fdiv_rn(mmin, c.s));
-  c.bias = kRoundMagicBits + c.zp;
   c.r = __fdiv_rn(1.0f, c.s);
-  c.fast = (c.s >= 0x1p-60f) && (c.s <= 0x1p60f);
+  c.nz2 = (static_cast<uint32_t>(-c.zp) & 0xffffu) * 0x10001u;
+  c.qm2 = static_cast<uint32_t>(c.qmax) * 0x10001u;
+  // rint(m / s) <= zp + qmax + 1 must stay a positive 16-bit integer for the packed steps
+  c.fast = (c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && (c.zp < 32000);
   return c;
 }
 
+// Code of one magnitude (scalar form: boundary checks only).
 template <int MODE>
 __device__ __forceinline__ int code_of(float m, const Level& c) {
   int k;
   if (MODE == kFast) {
-    k = __float_as_int(fmaf(m, c.r, kRoundMagic)) - c.bias;
-  } else if (MODE == kRefined) {
-    const float q0 = __fmul_rn(m, c.r);
-    const float q = fmaf(fmaf(-q0, c.s, m), c.r, q0);  // = fl(m / s)
-    k = __float_as_int(__fadd_rn(q, kRoundMagic)) - c.bias;
+    k = (__float_as_int(fmaf(m, c.r, kRoundMagic)) & 0xffff) - c.zp;
   } else {
     k = __float2int_rn(__fdiv_rn(m, c.s)) - c.zp;
   }
   return __vimin_s32_relu(k, c.qmax);  // clamp to [0, qmax]
+}
+
+// Codes of the two elements of a 16-bit pair (sign bits ignored), as two 16-bit integers.
+template <bool BF16, int MODE>
+__device__ __forceinline__ uint32_t codes2(uint32_t x, const Level& c) {
+  using E = Elem<BF16>;
+  const float lo = fabsf(E::lo_f32(x)), hi = fabsf(E::hi_f32(x));
+  if (MODE == kDivide) {
+    const int klo = __vimin_s32_relu(__float2int_rn(__fdiv_rn(lo, c.s)) - c.zp, c.qmax);
+    const int khi = __vimin_s32_relu(__float2int_rn(__fdiv_rn(hi, c.s)) - c.zp, c.qmax);
+    return static_cast<uint32_t>(klo) | (static_cast<uint32_t>(khi) << 16);
+  }
+  float tlo, thi;
+  if (MODE == kFast) {
+    tlo = fmaf(lo, c.r, kRoundMagic);
+    thi = fmaf(hi, c.r, kRoundMagic);
+  } else {
+    const float q0 = __fmul_rn(lo, c.r), q1 = __fmul_rn(hi, c.r);
+    tlo = __fadd_rn(fmaf(fmaf(-q0, c.s, lo), c.r, q0), kRoundMagic);  // fl(lo / s), then to an integer
+    thi = __fadd_rn(fmaf(fmaf(-q1, c.s, hi), c.r, q1), kRoundMagic);
+  }
+  // the low 16 bits of 1.5 * 2^23 + k are k itself
+  const uint32_t k2 = __byte_perm(__float_as_uint(tlo), __float_as_uint(thi), 0x5410);
+  return __viaddmin_s16x2_relu(k2, c.nz2, c.qm2);  // clamp(k - zp, 0, qmax) in both halves
 }
 
 // Does the fast path disagree with the true division for a 16-bit value next to rounding
@@ -119,14 +155,15 @@ __device__ __forceinline__ bool levels_disagree(const Level* first, const Level&
   return __any_sync(kFull, bad);
 }
 
-// Numerator of Algorithm 1's distortion for one row: sum |(q0 >> sh) - q|, whole warp.
+// Pass B. Numerator of Algorithm 1's distortion for one row: sum |(q0 >> sh) - q|, whole warp.
 template <bool BF16, int MODE>
-__device__ __forceinline__ int distortion(const uint4* row, const EncodeParams& p, uint32_t thr2, const Level& top,
-                                          const Level& low, int sh, uint32_t lane) {
-  using E = Elem<BF16>;
+__device__ __forceinline__ int distortion(const uint4* row, const EncodeParams& p, const Level& top, const Level& low,
+                                          int sh, uint32_t lane) {
+  const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
   uint32_t S = 0;
   for (uint32_t u = lane; u < p.units; u += 32) {
     const uint32_t rot = (u >> 1) & 3u;
+    uint32_t S2 = 0;  // two 16-bit partial sums: at most 16 * 127 each per unit
 #pragma unroll
     for (uint32_t j = 0; j < 4; ++j) {
       const uint32_t cidx = 4u * u + ((j + rot) & 3u);
@@ -135,50 +172,60 @@ __device__ __forceinline__ int distortion(const uint4* row, const EncodeParams& 
       const uint32_t x[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint32_t a = x[i] & 0x7fff7fffu;
-        const uint32_t m2 = a & ~E::geu_mask(a, thr2);
-        const float mlo = E::lo_f32(m2), mhi = E::hi_f32(m2);
-        S = __sad(code_of<MODE>(mlo, top) >> sh, code_of<MODE>(mlo, low), S);
-        S = __sad(code_of<MODE>(mhi, top) >> sh, code_of<MODE>(mhi, low), S);
+        const uint32_t a = (codes2<BF16, MODE>(x[i], top) >> sh) & shmask;
+        const uint32_t q = codes2<BF16, MODE>(x[i], low);
+        S2 += __vimax3_s16x2(a, q, q) - __vimin3_s16x2(a, q, q);
       }
     }
+    S += (S2 & 0xffffu) + (S2 >> 16);
   }
   return static_cast<int>(__reduce_add_sync(kFull, S));
 }
 
-// Codes of the row at the chosen level, packed as bytes (code << 1 | sign), transposed into
-// bit-planes and stored: plane 0 = sign, plane 1 + k = bit k of the code.
+// Pass C. Codes of the row at the chosen level as bytes (code << 1 | sign), transposed into
+// bit-planes (plane 0 = sign, plane 1 + k = bit k of the code) and written over the front of the
+// slot: group g's b* words go to words g * b* .. g * b* + b* - 1.
 template <bool BF16, int MODE>
-__device__ __forceinline__ void pack_row(const uint4* row, const EncodeParams& p, uint32_t thr2, const Level& lv,
-                                         int bstar, uint32_t* wdst, uint32_t lane) {
-  using E = Elem<BF16>;
-  for (uint32_t u = lane; u < p.units; u += 32) {
+__device__ __forceinline__ void pack_row(uint4* row, const EncodeParams& p, const Level& lv, int bstar, uint32_t lane) {
+  uint32_t* out = reinterpret_cast<uint32_t*>(row);
+  for (uint32_t base = 0; base < p.units; base += 32) {
+    const uint32_t u = base + lane;
     const uint32_t rot = (u >> 1) & 3u;
+    uint4 c[4];
+#pragma unroll
+    for (uint32_t j = 0; j < 4; ++j) {
+      const uint32_t cidx = 4u * u + ((j + rot) & 3u);
+      c[j] = (u < p.units && cidx < p.chunks) ? row[cidx] : make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncwarp();  // all 32 groups are in registers before any of them is overwritten
+    if (u >= p.units) continue;
     uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #pragma unroll
     for (uint32_t j = 0; j < 4; ++j) {
       const uint32_t cc = (j + rot) & 3u;
-      const uint32_t cidx = 4u * u + cc;
-      if (cidx >= p.chunks) continue;
-      const uint4 c = row[cidx];
-      const uint32_t x[4] = {c.x, c.y, c.z, c.w};
-      const uint32_t shift = 8u * cc;
+      // selectors that put byte 0 / byte 2 of the second operand into byte cc of the first
+      const uint32_t keep_sel = 0x3210u & ~(0xfu << (4u * cc));
+      const uint32_t sel_lo = keep_sel | (4u << (4u * cc)), sel_hi = keep_sel | (6u << (4u * cc));
+      const uint32_t x[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint32_t a = x[i] & 0x7fff7fffu;
-        const uint32_t mk = E::geu_mask(a, thr2);
-        const uint32_t keep = x[i] & ~mk;  // inliers keep sign and magnitude, outlier slots become +0
-        const uint32_t m2 = keep & 0x7fff7fffu;
-        const uint32_t blo = (static_cast<uint32_t>(code_of<MODE>(E::lo_f32(m2), lv)) << 1) | ((keep >> 15) & 1u);
-        const uint32_t bhi = (static_cast<uint32_t>(code_of<MODE>(E::hi_f32(m2), lv)) << 1) | (keep >> 31);
-        r[2 * i] |= blo << shift;
-        r[2 * i + 1] |= bhi << shift;
+        const uint32_t b2 = codes2<BF16, MODE>(x[i], lv) * 2u + ((x[i] >> 15) & 0x00010001u);
+        r[2 * i] = __byte_perm(r[2 * i], b2, sel_lo);
+        r[2 * i + 1] = __byte_perm(r[2 * i + 1], b2, sel_hi);
       }
     }
     transpose8x32(r);
+    uint32_t* dst = out + static_cast<size_t>(u) * bstar;
+    if (bstar == 8) {
+      reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[0], r[1], r[2], r[3]);
+      reinterpret_cast<uint4*>(dst)[1] = make_uint4(r[4], r[5], r[6], r[7]);
+    } else if (bstar == 4) {
+      reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[0], r[1], r[2], r[3]);
+    } else {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      if (k < bstar) wdst[static_cast<size_t>(k) * p.lay.wpp + u] = r[k];
+      for (int k = 0; k < 8; ++k) {
+        if (k < bstar) dst[k] = r[k];
+      }
     }
   }
 }
@@ -187,18 +234,24 @@ __device__ __forceinline__ unsigned long long pack_desc(uint32_t tag, uint32_t v
   return (static_cast<unsigned long long>(tag) << 32) | value;
 }
 
-// Decoupled look-back, run by one full warp for its own tile.
+// Decoupled look-back over the tile descriptors.
 // Descriptor of tile t: (generation * 4 + flag) << 32 | payload.  An AGGREGATE payload carries the
 // tile's own sizes, (outliers << 15) | plane words; a PREFIX payload carries the inclusive prefix
 // of plane words, and the inclusive prefix of outliers sits in prefix_outl[t], stored before the
 // descriptor with a fence between the two.
+__device__ __forceinline__ void publish_aggregate(const EncodeParams& p, uint32_t gen4, uint32_t tile, uint32_t agg_w,
+                                                  uint32_t agg_o, uint32_t lane) {
+  if (tile > 0 && lane == 0) st_relaxed_u64(p.desc + tile, pack_desc(gen4 | kFlagAggregate, (agg_o << 15) | agg_w));
+}
+
+// Run by one full warp for its own tile, after publish_aggregate: walk back to the nearest
+// published prefix, then publish this tile's own.
 // Returns TSQ_OK, TSQ_ERR_TIMEOUT (gave up) or -1 when a predecessor has aborted.
-__device__ int lookback(const EncodeParams& p, uint32_t gen4, uint32_t tile, uint32_t agg_w, uint32_t agg_o,
-                        uint32_t lane, uint32_t* excl_w, uint32_t* excl_o) {
+__device__ int resolve_prefix(const EncodeParams& p, uint32_t gen4, uint32_t tile, uint32_t agg_w, uint32_t agg_o,
+                              uint32_t lane, uint32_t* excl_w, uint32_t* excl_o) {
   uint32_t base_w = 0, base_o = 0;  // prefix found at the end of the walk
   uint32_t part_w = 0, part_o = 0;  // this lane's share of the aggregates walked over
   if (tile > 0) {
-    if (lane == 0) st_relaxed_u64(p.desc + tile, pack_desc(gen4 | kFlagAggregate, (agg_o << 15) | agg_w));
     int pos = static_cast<int>(tile) - 1;  // nearest tile not yet accounted for
     uint32_t polls = 0;
     bool done = false;
@@ -245,7 +298,7 @@ __device__ int lookback(const EncodeParams& p, uint32_t gen4, uint32_t tile, uin
         pos -= consumed;
         if (consumed == 0) {
           if (++polls > kLookbackPollLimit) return TSQ_ERR_TIMEOUT;
-          __nanosleep(polls < 8u ? 100u : 400u);
+          __nanosleep(polls < 8u ? 200u : 1000u);
         }
       }
     }
@@ -280,56 +333,67 @@ __device__ void write_header(const EncodeParams& p, unsigned long long total_wor
 }
 
 // All passes of the method on one row held in shared memory.  Returns TSQ_OK, TSQ_ERR_TIMEOUT,
-// or 0xffffffff when a predecessor aborted (nothing further to report).
+// or 0xffffffff when a predecessor aborted (nothing further to report).  *stored tells the caller
+// that a bulk store out of the slot is in flight.
 template <bool BF16>
-__device__ uint32_t encode_row(const EncodeParams& p, uint32_t gen4, uint32_t tile, const uint4* row,
-                               uint16_t* s_list, uint32_t lane) {
+__device__ uint32_t encode_row(const EncodeParams& p, uint32_t gen4, uint32_t tile, uint4* row, uint32_t* stash,
+                               uint32_t lane, bool* stored) {
   using E = Elem<BF16>;
   const uint32_t thr2 = p.thr16 * 0x10001u;
-  const uint16_t* row16 = reinterpret_cast<const uint16_t*>(row);
+  uint16_t* row16 = reinterpret_cast<uint16_t*>(row);
 
-  // ---- pass A: threshold split, min / max of the magnitudes, list of units holding outliers ----
-  uint32_t mn2 = E::kInfPattern * 0x10001u, mx2 = 0u, n_list = 0u;
+  // ---- pass A: threshold split, min / max of the inlier magnitudes, outliers to the stash ----
+  uint32_t mn2 = E::kInfPattern * 0x10001u, mx2 = 0u, row_cnt = 0u;
   for (uint32_t base = 0; base < p.units; base += 32) {
     const uint32_t u = base + lane;
-    uint32_t any = 0u;
+    uint32_t bitmap = 0u;  // bit e: element 32u + e is an outlier
     if (u < p.units) {
       const uint32_t rot = (u >> 1) & 3u;
 #pragma unroll
       for (uint32_t j = 0; j < 4; ++j) {
-        const uint32_t cidx = 4u * u + ((j + rot) & 3u);
+        const uint32_t cc = (j + rot) & 3u;
+        const uint32_t cidx = 4u * u + cc;
         if (cidx >= p.chunks) continue;
         const uint4 c = row[cidx];
         const uint32_t x[4] = {c.x, c.y, c.z, c.w};
+        uint32_t acc = 0u;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint32_t a = x[i] & 0x7fff7fffu;
-          const uint32_t mk = E::geu_mask(a, thr2);
+          const uint32_t mk = E::geu_mask(a, thr2);  // 0xffff in each half with |x| >= tau, NaN included
           const uint32_t m2 = a & ~mk;
           mx2 = E::max2(mx2, m2);
           mn2 = E::min2(mn2, m2);
-          any |= mk;
+          acc |= mk & ((1u << (2 * i)) | (1u << (17 + 2 * i)));
         }
+        bitmap |= ((acc | (acc >> 16)) & 0xffu) << (8u * cc);
       }
     }
-    const uint32_t bal = __ballot_sync(kFull, any != 0u);
+    const uint32_t bal = __ballot_sync(kFull, bitmap != 0u);
     if (bal != 0u) {
-      if (any != 0u) s_list[n_list + __popc(bal & ((1u << lane) - 1u))] = static_cast<uint16_t>(u);
-      n_list += __popc(bal);
+      // groups holding outliers, in ascending order; one element per lane
+      uint32_t rest = bal;
+      while (rest != 0u) {
+        const uint32_t src = static_cast<uint32_t>(__ffs(rest) - 1);
+        rest &= rest - 1u;
+        const uint32_t bm = __shfl_sync(kFull, bitmap, src);
+        if ((bm >> lane) & 1u) {
+          const uint32_t at = row_cnt + __popc(bm & ((1u << lane) - 1u));
+          const uint32_t e = 32u * (base + src) + lane;
+          if (at < p.stash_cap) stash[at] = (e << 16) | row16[e];
+        }
+        row_cnt += __popc(bm);
+      }
+      __syncwarp();  // the stash has the original patterns before their slots are cleared
+      while (bitmap != 0u) {
+        row16[32u * u + static_cast<uint32_t>(__ffs(bitmap) - 1)] = 0;  // T_below holds +0 there
+        bitmap &= bitmap - 1u;
+      }
     }
   }
   const uint32_t pmin = __reduce_min_sync(kFull, min(mn2 & 0xffffu, mn2 >> 16));
   const uint32_t pmax = __reduce_max_sync(kFull, max(mx2 & 0xffffu, mx2 >> 16));
   __syncwarp();
-
-  // outliers of the row: one listed unit at a time, one element per lane
-  uint32_t row_cnt = 0u;
-  for (uint32_t k = 0; k < n_list; ++k) {
-    const uint32_t e = 32u * s_list[k] + lane;
-    // patterns of non-negative values order like the values; NaN patterns sort above +Inf
-    const bool out = e < p.hidden && (row16[e] & 0x7fffu) >= p.thr16;
-    row_cnt += __popc(__ballot_sync(kFull, out));
-  }
 
   // ---- Algorithm 1: descend the candidate list while the distortion stays within tolerance ----
   const float mmin = E::pattern_f32(pmin), mmax = E::pattern_f32(pmax);
@@ -349,21 +413,44 @@ __device__ uint32_t encode_row(const EncodeParams& p, uint32_t gen4, uint32_t ti
       if (levels_disagree<BF16>(top_checked ? nullptr : &top, low, pmin, pmax, lane)) mode = kRefined;
       top_checked = true;
     }
-    const int S = mode == kFast      ? distortion<BF16, kFast>(row, p, thr2, top, low, sh, lane)
-                  : mode == kRefined ? distortion<BF16, kRefined>(row, p, thr2, top, low, sh, lane)
-                                     : distortion<BF16, kDivide>(row, p, thr2, top, low, sh, lane);
+    const int S = mode == kFast      ? distortion<BF16, kFast>(row, p, top, low, sh, lane)
+                  : mode == kRefined ? distortion<BF16, kRefined>(row, p, top, low, sh, lane)
+                                     : distortion<BF16, kDivide>(row, p, top, low, sh, lane);
     if (S > p.s_max) break;  // delta > Delta: keep the last level that passed
     bstar = b;
     best = low;
   }
 
+  // ---- this row's sizes are known: let the rows behind it see them, then pack ----
+  const uint32_t agg_w = static_cast<uint32_t>(bstar) * p.lay.wpp;
+  publish_aggregate(p, gen4, tile, agg_w, row_cnt, lane);
+  if (mode == kFast) {
+    pack_row<BF16, kFast>(row, p, best, bstar, lane);
+  } else if (mode == kRefined) {
+    pack_row<BF16, kRefined>(row, p, best, bstar, lane);
+  } else {
+    pack_row<BF16, kDivide>(row, p, best, bstar, lane);
+  }
+  fence_proxy_async_smem();  // the packed words are about to be read by the bulk-copy engine
+  __syncwarp();
+
   // ---- placement: exclusive prefix sums over the tokens before this one ----
   uint32_t word_off = 0, out_base = 0;
-  const uint32_t agg_w = static_cast<uint32_t>(bstar) * p.lay.wpp;
-  const int st = lookback(p, gen4, tile, agg_w, row_cnt, lane, &word_off, &out_base);
+  const int st = resolve_prefix(p, gen4, tile, agg_w, row_cnt, lane, &word_off, &out_base);
   if (st != TSQ_OK) {
     if (lane == 0) st_relaxed_u64(p.desc + tile, pack_desc(gen4 | kFlagAbort, 0u));
     return st < 0 ? 0xffffffffu : static_cast<uint32_t>(st);
+  }
+  uint32_t* wdst = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_words) + word_off;
+  if (p.bulk_store) {
+    if (lane == 0) {
+      bulk_s2g(wdst, row, agg_w * 4u);
+      bulk_commit();
+    }
+    *stored = true;
+  } else {  // word counts that are not multiples of 16 bytes: plain stores
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(row);
+    for (uint32_t w = lane; w < agg_w; w += 32) wdst[w] = src[w];
   }
   if (lane == 0) {
     reinterpret_cast<uint8_t*>(p.blob + p.lay.off_bits)[tile] = static_cast<uint8_t>(bstar);
@@ -379,35 +466,39 @@ __device__ uint32_t encode_row(const EncodeParams& p, uint32_t gen4, uint32_t ti
     o_out_ptr[tile + 1] = out_base + row_cnt;
   }
 
-  // ---- pack the planes of the chosen level ----
-  uint32_t* wdst = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_words) + word_off;
-  if (mode == kFast) {
-    pack_row<BF16, kFast>(row, p, thr2, best, bstar, wdst, lane);
-  } else if (mode == kRefined) {
-    pack_row<BF16, kRefined>(row, p, thr2, best, bstar, wdst, lane);
-  } else {
-    pack_row<BF16, kDivide>(row, p, thr2, best, bstar, wdst, lane);
-  }
-
   // ---- CSR entries of T_above: ascending columns, original patterns ----
   if (row_cnt != 0u) {
     uint32_t* o_outl = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_outl);
-    unsigned long long pos = out_base;
     bool overflow = false;
-    for (uint32_t k = 0; k < n_list; ++k) {
-      const uint32_t e = 32u * s_list[k] + lane;
-      const uint32_t raw = e < p.hidden ? row16[e] : 0u;
-      const bool out = e < p.hidden && (raw & 0x7fffu) >= p.thr16;
-      const uint32_t bal = __ballot_sync(kFull, out);
-      if (out) {
-        const unsigned long long at = pos + __popc(bal & ((1u << lane) - 1u));
+    if (row_cnt <= p.stash_cap) {
+      for (uint32_t i = lane; i < row_cnt; i += 32) {
+        const unsigned long long at = static_cast<unsigned long long>(out_base) + i;
         if (at < p.lay.outlier_capacity) {
-          o_outl[at] = (e << 16) | raw;
+          o_outl[at] = stash[i];
         } else {
           overflow = true;
         }
       }
-      pos += __popc(bal);
+    } else {
+      // more outliers than the stash holds: take them from the input row in global memory again
+      const uint16_t* xrow = p.x + static_cast<size_t>(tile) * p.hidden;
+      unsigned long long pos = out_base;
+      for (uint32_t g = 0; g < p.units; ++g) {
+        const uint32_t e = 32u * g + lane;
+        const uint32_t raw = e < p.hidden ? xrow[e] : 0u;
+        // patterns of non-negative values order like the values; NaN patterns sort above +Inf
+        const bool out = e < p.hidden && (raw & 0x7fffu) >= p.thr16;
+        const uint32_t bal = __ballot_sync(kFull, out);
+        if (out) {
+          const unsigned long long at = pos + __popc(bal & ((1u << lane) - 1u));
+          if (at < p.lay.outlier_capacity) {
+            o_outl[at] = (e << 16) | raw;
+          } else {
+            overflow = true;
+          }
+        }
+        pos += __popc(bal);
+      }
     }
     if (__any_sync(kFull, overflow) && lane == 0) {
       atomicCAS(&p.ws->err, 0u, static_cast<uint32_t>(TSQ_ERR_OUTLIER_OVERFLOW));
@@ -426,8 +517,8 @@ __global__ void __launch_bounds__(kEncMaxWarps * 32, 1) encode_kernel(const Enco
 
   if (warp < p.active_warps) {
     unsigned char* slot = smem_dyn + static_cast<size_t>(warp) * p.warp_stride;
-    const uint4* row = reinterpret_cast<const uint4*>(slot);
-    uint16_t* s_list = reinterpret_cast<uint16_t*>(slot + p.row_stride);
+    uint4* row = reinterpret_cast<uint4*>(slot);
+    uint32_t* stash = reinterpret_cast<uint32_t*>(slot + p.row_stride);
     uint64_t* bar = &s_bar[warp];
     if (lane == 0) {
       mbar_init(bar, 1);
@@ -436,19 +527,22 @@ __global__ void __launch_bounds__(kEncMaxWarps * 32, 1) encode_kernel(const Enco
     __syncwarp();
 
     uint32_t parity = 0;
+    bool stored = false;  // a bulk store out of the slot may still be reading it
     for (;;) {
       uint32_t tile = 0;
       if (lane == 0) tile = atomicAdd(&p.ws->ticket, 1u);
       tile = __shfl_sync(kFull, tile, 0);
       if (tile >= p.tokens) break;
       if (lane == 0) {
+        if (stored) bulk_wait_read_all();
         mbar_arrive_expect_tx(bar, p.row_bytes);
         bulk_g2s(slot, p.x + static_cast<size_t>(tile) * p.hidden, p.row_bytes, bar);
       }
+      stored = false;
       uint32_t err = TSQ_OK;
       if (__all_sync(kFull, mbar_wait_bounded(bar, parity, kCopyPollLimit))) {
         parity ^= 1u;
-        err = encode_row<BF16>(p, gen4, tile, row, s_list, lane);
+        err = encode_row<BF16>(p, gen4, tile, row, stash, lane, &stored);
       } else {
         // the copy did not land in time: tell the rows behind, give it one more bounded chance to land
         err = TSQ_ERR_TIMEOUT;
@@ -461,6 +555,7 @@ __global__ void __launch_bounds__(kEncMaxWarps * 32, 1) encode_kernel(const Enco
       }
       __syncwarp();  // every lane is done with the slot before the next copy overwrites it
     }
+    if (lane == 0) bulk_wait_all();  // the slot must outlive the stores that read it
   }
 
   // ---- the CTA that finishes last publishes the status and re-arms the workspace ----

@@ -84,7 +84,9 @@ struct EncodeParams {
   int32_t bits[8];
   int32_t s_max;                             // floor(delta * H), clamped to [-1, INT32_MAX]
   uint32_t row_bytes;                        // bytes of one input row
-  uint32_t row_stride, warp_stride;          // shared memory: row slot, and row slot + unit list, per warp
+  uint32_t row_stride, warp_stride;          // shared memory per warp: row slot, and row slot + outlier stash
+  uint32_t stash_cap;                        // entries of the outlier stash
+  uint32_t bulk_store;                       // 1: every token's plane words are a multiple of 16 bytes
   uint32_t active_warps;                     // warps of each CTA that take rows
   uint32_t dtype;
   float tau, delta;

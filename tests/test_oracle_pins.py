@@ -40,16 +40,16 @@ def f32_to_raw(v, dtype):
 
 
 def unpack_planes(words_row, b, hidden):
-    """Independent scalar reader of one token's bit-planes: returns (sign[H], code[H])."""
-    wpp = (hidden + 31) // 32
+    """Independent scalar reader of one token's bit-planes: returns (sign[H], code[H]).
+    Group g (elements 32g .. 32g+31) owns words g*b .. g*b+b-1: plane 0 = sign, plane 1+k = code bit k."""
     sign = np.zeros(hidden, np.int64)
     code = np.zeros(hidden, np.int64)
     for j in range(hidden):
-        w, i = divmod(j, 32)
-        sign[j] = (int(words_row[w]) >> i) & 1
+        g, i = divmod(j, 32)
+        sign[j] = (int(words_row[g * b]) >> i) & 1
         c = 0
         for k in range(b - 1):
-            c |= ((int(words_row[(1 + k) * wpp + w]) >> i) & 1) << k
+            c |= ((int(words_row[g * b + 1 + k]) >> i) & 1) << k
         code[j] = c
     return sign, code
 
@@ -354,7 +354,7 @@ def test_blob_layout_offsets_and_restore(dtype, hidden):
         # pad bits of the last word are zero in every plane
         if hidden % 32:
             mask = np.uint32((0xffffffff << (hidden % 32)) & 0xffffffff)
-            assert np.all(words_row.reshape(b, wpp)[:, -1] & mask == 0)
+            assert np.all(words_row.reshape(wpp, b)[-1, :] & mask == 0)
         # inlier error bound after the cast: s/2 + half a 16-bit ulp of the restored value
         inl = ~out[t]
         s = float(sec["scale"][t])
