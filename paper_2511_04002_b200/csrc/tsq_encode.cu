@@ -50,7 +50,8 @@
 namespace tsq {
 namespace {
 
-constexpr float kRoundMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer, ties to even
+constexpr float kRoundMagic = 8388608.0f;  // 2^23: adding it to 0 <= y < 2^23 rounds y to an integer, ties to even
+constexpr uint32_t kRoundMagicHi = 0x4B00u;  // upper 16 bits of the pattern of 2^23
 constexpr uint32_t kLookbackPollLimit = 1u << 20;
 constexpr uint32_t kCopyPollLimit = 1u << 20;
 constexpr int kLookbackDepth = 8;  // descriptors each lane reads per look-back step
@@ -61,7 +62,7 @@ struct Level {
   float r;       // fl(1 / s)
   int zp;        // zero-point rint(m_min / s)
   int qmax;      // 2^(b-1) - 1
-  uint32_t nz2;  // -zp in both 16-bit halves
+  uint32_t nz2;  // -zp in the low half, -zp - kRoundMagicHi in the high half (see codes2)
   uint32_t qm2;  // qmax in both 16-bit halves
   bool fast;     // scale and zero-point in the range where the FMA paths are provably safe
 };
@@ -75,10 +76,10 @@ __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
   c.s = range > 0.0f ? __fdiv_rn(range, static_cast<float>(c.qmax)) : (mmax > 0.0f ? mmax : 1.0f);
   c.zp = __float2int_rn(__fdiv_rn(mmin, c.s));
   c.r = __fdiv_rn(1.0f, c.s);
-  c.nz2 = (static_cast<uint32_t>(-c.zp) & 0xffffu) * 0x10001u;
+  c.nz2 = (static_cast<uint32_t>(-c.zp) & 0xffffu) | (static_cast<uint32_t>(-c.zp - static_cast<int>(kRoundMagicHi)) << 16);
   c.qm2 = static_cast<uint32_t>(c.qmax) * 0x10001u;
-  // rint(m / s) <= zp + qmax + 1 must stay a positive 16-bit integer for the packed steps
-  c.fast = (c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && (c.zp < 32000);
+  // rint(m / s) <= zp + qmax + 1 must stay a small positive 16-bit integer for the packed steps
+  c.fast = (c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && (c.zp < 12000);
   return c;
 }
 
@@ -113,8 +114,9 @@ __device__ __forceinline__ uint32_t codes2(uint32_t x, const Level& c) {
     tlo = __fadd_rn(fmaf(fmaf(-q0, c.s, lo), c.r, q0), kRoundMagic);  // fl(lo / s), then to an integer
     thi = __fadd_rn(fmaf(fmaf(-q1, c.s, hi), c.r, q1), kRoundMagic);
   }
-  // the low 16 bits of 1.5 * 2^23 + k are k itself
-  const uint32_t k2 = __byte_perm(__float_as_uint(tlo), __float_as_uint(thi), 0x5410);
+  // pattern of 2^23 + k = 0x4B000000 + k.  thi * 2^16 + tlo (mod 2^32) = (0x4B00 + k_lo's carry-free
+  // neighbour k_hi) << 16 | k_lo; the constant in the high half is taken off together with zp.
+  const uint32_t k2 = __float_as_uint(thi) * 65536u + __float_as_uint(tlo);
   return __viaddmin_s16x2_relu(k2, c.nz2, c.qm2);  // clamp(k - zp, 0, qmax) in both halves
 }
 
@@ -155,76 +157,96 @@ __device__ __forceinline__ bool levels_disagree(const Level* first, const Level&
   return __any_sync(kFull, bad);
 }
 
+__device__ __forceinline__ uint32_t max_s16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.s16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ uint32_t min_s16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("min.s16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
 // Pass B. Numerator of Algorithm 1's distortion for one row: sum |(q0 >> sh) - q|, whole warp.
+// The terms are non-negative, so the pass stops as soon as the running sum exceeds s_max: the
+// returned value is then only known to be > s_max, which is all the caller asks.
 template <bool BF16, int MODE>
 __device__ __forceinline__ int distortion(const uint4* row, const EncodeParams& p, const Level& top, const Level& low,
                                           int sh, uint32_t lane) {
   const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
   uint32_t S = 0;
-  for (uint32_t u = lane; u < p.units; u += 32) {
-    const uint32_t rot = (u >> 1) & 3u;
+  int total = 0;
+  for (uint32_t base = 0; base < p.units; base += 32) {
+    const uint32_t u = base + lane;
     uint32_t S2 = 0;  // two 16-bit partial sums: at most 16 * 127 each per unit
+    if (u < p.units) {
 #pragma unroll
-    for (uint32_t j = 0; j < 4; ++j) {
-      const uint32_t cidx = 4u * u + ((j + rot) & 3u);
-      if (cidx >= p.chunks) continue;
-      const uint4 c = row[cidx];
-      const uint32_t x[4] = {c.x, c.y, c.z, c.w};
+      for (uint32_t j = 0; j < 4; ++j) {
+        const uint32_t cidx = 4u * u + j;
+        if (cidx >= p.chunks) continue;
+        const uint4 c = row[cidx];
+        const uint32_t x[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t a = (codes2<BF16, MODE>(x[i], top) >> sh) & shmask;
-        const uint32_t q = codes2<BF16, MODE>(x[i], low);
-        S2 += __vimax3_s16x2(a, q, q) - __vimin3_s16x2(a, q, q);
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t a = (codes2<BF16, MODE>(x[i], top) >> sh) & shmask;
+          const uint32_t q = codes2<BF16, MODE>(x[i], low);
+          S2 += max_s16x2(a, q) - min_s16x2(a, q);
+        }
       }
     }
     S += (S2 & 0xffffu) + (S2 >> 16);
+    total = static_cast<int>(__reduce_add_sync(kFull, S));
+    if (total > p.s_max) break;
   }
-  return static_cast<int>(__reduce_add_sync(kFull, S));
+  return total;
 }
 
-// Pass C. Codes of the row at the chosen level as bytes (code << 1 | sign), transposed into
-// bit-planes (plane 0 = sign, plane 1 + k = bit k of the code) and written over the front of the
-// slot: group g's b* words go to words g * b* .. g * b* + b* - 1.
+// Pass C. Codes of the row at the chosen level as bytes (code | sign << 7), transposed into
+// bit-planes and written over the front of the slot: group g's b* words go to words
+// g * b* .. g * b* + b* - 1, plane 0 = sign, plane 1 + k = bit k of the code.
 template <bool BF16, int MODE>
 __device__ __forceinline__ void pack_row(uint4* row, const EncodeParams& p, const Level& lv, int bstar, uint32_t lane) {
   uint32_t* out = reinterpret_cast<uint32_t*>(row);
   for (uint32_t base = 0; base < p.units; base += 32) {
     const uint32_t u = base + lane;
-    const uint32_t rot = (u >> 1) & 3u;
     uint4 c[4];
 #pragma unroll
     for (uint32_t j = 0; j < 4; ++j) {
-      const uint32_t cidx = 4u * u + ((j + rot) & 3u);
+      const uint32_t cidx = 4u * u + j;
       c[j] = (u < p.units && cidx < p.chunks) ? row[cidx] : make_uint4(0u, 0u, 0u, 0u);
     }
     __syncwarp();  // all 32 groups are in registers before any of them is overwritten
     if (u >= p.units) continue;
-    uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    // b2[j][i]: bytes of elements 8j + 2i (byte 0) and 8j + 2i + 1 (byte 2)
+    uint32_t b2[4][4];
 #pragma unroll
     for (uint32_t j = 0; j < 4; ++j) {
-      const uint32_t cc = (j + rot) & 3u;
-      // selectors that put byte 0 / byte 2 of the second operand into byte cc of the first
-      const uint32_t keep_sel = 0x3210u & ~(0xfu << (4u * cc));
-      const uint32_t sel_lo = keep_sel | (4u << (4u * cc)), sel_hi = keep_sel | (6u << (4u * cc));
       const uint32_t x[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t b2 = codes2<BF16, MODE>(x[i], lv) * 2u + ((x[i] >> 15) & 0x00010001u);
-        r[2 * i] = __byte_perm(r[2 * i], b2, sel_lo);
-        r[2 * i + 1] = __byte_perm(r[2 * i + 1], b2, sel_hi);
-      }
+      for (int i = 0; i < 4; ++i) b2[j][i] = codes2<BF16, MODE>(x[i], lv) | ((x[i] >> 8) & 0x00800080u);
     }
-    transpose8x32(r);
+    // r[i] byte c = element 8c + i
+    uint32_t r[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t e = b2[1][i] * 256u + b2[0][i];  // bytes: 8*0+2i, 8*1+2i, 8*0+2i+1, 8*1+2i+1
+      const uint32_t f = b2[3][i] * 256u + b2[2][i];  // the same for chunks 2 and 3
+      r[2 * i] = __byte_perm(e, f, 0x5410);
+      r[2 * i + 1] = __byte_perm(e, f, 0x7632);
+    }
+    transpose8x32(r);  // r[k] = bit k of every byte: k < 7 code bits, k = 7 signs
     uint32_t* dst = out + static_cast<size_t>(u) * bstar;
     if (bstar == 8) {
-      reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[0], r[1], r[2], r[3]);
-      reinterpret_cast<uint4*>(dst)[1] = make_uint4(r[4], r[5], r[6], r[7]);
+      reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[7], r[0], r[1], r[2]);
+      reinterpret_cast<uint4*>(dst)[1] = make_uint4(r[3], r[4], r[5], r[6]);
     } else if (bstar == 4) {
-      reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[0], r[1], r[2], r[3]);
+      reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[7], r[0], r[1], r[2]);
     } else {
+      dst[0] = r[7];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        if (k < bstar) dst[k] = r[k];
+      for (int k = 0; k < 7; ++k) {
+        if (k < bstar - 1) dst[1 + k] = r[k];
       }
     }
   }
@@ -297,8 +319,17 @@ __device__ int resolve_prefix(const EncodeParams& p, uint32_t gen4, uint32_t til
       if (!done) {
         pos -= consumed;
         if (consumed == 0) {
-          if (++polls > kLookbackPollLimit) return TSQ_ERR_TIMEOUT;
-          __nanosleep(polls < 8u ? 200u : 1000u);
+          // tile `pos` has published nothing yet: watch that one descriptor until it does
+          for (;;) {
+            uint32_t ready = 0u;
+            if (lane == 0) {
+              const uint32_t tag = static_cast<uint32_t>(ld_relaxed_u64(p.desc + pos) >> 32);
+              ready = ((tag & ~3u) == gen4 && (tag & 3u) != 0u) ? 1u : 0u;
+            }
+            if (__shfl_sync(kFull, ready, 0) != 0u) break;
+            if (++polls > kLookbackPollLimit) return TSQ_ERR_TIMEOUT;
+            __nanosleep(polls < 16u ? 250u : 1000u);
+          }
         }
       }
     }
@@ -346,48 +377,50 @@ __device__ uint32_t encode_row(const EncodeParams& p, uint32_t gen4, uint32_t ti
   uint32_t mn2 = E::kInfPattern * 0x10001u, mx2 = 0u, row_cnt = 0u;
   for (uint32_t base = 0; base < p.units; base += 32) {
     const uint32_t u = base + lane;
-    uint32_t bitmap = 0u;  // bit e: element 32u + e is an outlier
+    uint32_t acc[4] = {0u, 0u, 0u, 0u};  // per chunk: bit 2i / bit 17 + 2i flag the low / high element of pair i
     if (u < p.units) {
-      const uint32_t rot = (u >> 1) & 3u;
 #pragma unroll
       for (uint32_t j = 0; j < 4; ++j) {
-        const uint32_t cc = (j + rot) & 3u;
-        const uint32_t cidx = 4u * u + cc;
+        const uint32_t cidx = 4u * u + j;
         if (cidx >= p.chunks) continue;
         const uint4 c = row[cidx];
         const uint32_t x[4] = {c.x, c.y, c.z, c.w};
-        uint32_t acc = 0u;
+        uint32_t m2[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint32_t a = x[i] & 0x7fff7fffu;
           const uint32_t mk = E::geu_mask(a, thr2);  // 0xffff in each half with |x| >= tau, NaN included
-          const uint32_t m2 = a & ~mk;
-          mx2 = E::max2(mx2, m2);
-          mn2 = E::min2(mn2, m2);
-          acc |= mk & ((1u << (2 * i)) | (1u << (17 + 2 * i)));
+          m2[i] = a & ~mk;
+          acc[j] |= mk & ((1u << (2 * i)) | (1u << (17 + 2 * i)));
         }
-        bitmap |= ((acc | (acc >> 16)) & 0xffu) << (8u * cc);
+        // patterns of non-negative values order like the values: integer min / max
+        mx2 = __vimax3_u16x2(mx2, m2[0], m2[1]);
+        mx2 = __vimax3_u16x2(mx2, m2[2], m2[3]);
+        mn2 = __vimin3_u16x2(mn2, m2[0], m2[1]);
+        mn2 = __vimin3_u16x2(mn2, m2[2], m2[3]);
       }
     }
-    const uint32_t bal = __ballot_sync(kFull, bitmap != 0u);
-    if (bal != 0u) {
-      // groups holding outliers, in ascending order; one element per lane
-      uint32_t rest = bal;
-      while (rest != 0u) {
-        const uint32_t src = static_cast<uint32_t>(__ffs(rest) - 1);
-        rest &= rest - 1u;
-        const uint32_t bm = __shfl_sync(kFull, bitmap, src);
-        if ((bm >> lane) & 1u) {
-          const uint32_t at = row_cnt + __popc(bm & ((1u << lane) - 1u));
-          const uint32_t e = 32u * (base + src) + lane;
-          if (at < p.stash_cap) stash[at] = (e << 16) | row16[e];
-        }
-        row_cnt += __popc(bm);
+    const uint32_t any = acc[0] | acc[1] | acc[2] | acc[3];
+    if (__ballot_sync(kFull, any != 0u) != 0u) {
+      uint32_t bitmap = 0u;  // bit e: element 32u + e is an outlier
+#pragma unroll
+      for (uint32_t j = 0; j < 4; ++j) bitmap |= ((acc[j] | (acc[j] >> 16)) & 0xffu) << (8u * j);
+      // where this lane's entries go: exclusive scan of the per-lane counts, columns stay ascending
+      const uint32_t cnt = __popc(bitmap);
+      uint32_t incl = cnt;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t n = __shfl_up_sync(kFull, incl, d);
+        if (lane >= static_cast<uint32_t>(d)) incl += n;
       }
-      __syncwarp();  // the stash has the original patterns before their slots are cleared
+      uint32_t at = row_cnt + incl - cnt;
+      row_cnt += __shfl_sync(kFull, incl, 31);
       while (bitmap != 0u) {
-        row16[32u * u + static_cast<uint32_t>(__ffs(bitmap) - 1)] = 0;  // T_below holds +0 there
+        const uint32_t e = 32u * u + static_cast<uint32_t>(__ffs(bitmap) - 1);
         bitmap &= bitmap - 1u;
+        if (at < p.stash_cap) stash[at] = (e << 16) | row16[e];
+        ++at;
+        row16[e] = 0;  // T_below holds +0 there
       }
     }
   }
