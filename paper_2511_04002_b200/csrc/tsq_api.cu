@@ -63,8 +63,7 @@ struct tsq_plan {
   int32_t s_max;
   uint32_t thr16;
   int threads;                      // decoder CTA size
-  uint32_t enc_row_stride, enc_warp_stride, enc_stash_cap;
-  int enc_warps;                    // warps per encoder CTA that fit in shared memory
+  int enc_threads, enc_upt;         // encoder CTA size and 32-element groups per thread
   int sms;
   size_t dec_smem;
   size_t workspace_bytes;
@@ -128,14 +127,12 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   p->thr16 = threshold_pattern(dtype, tau);
   p->threads = static_cast<int>(((p->units + 31u) / 32u) * 32u);
   if (p->threads > kMaxThreads) p->threads = kMaxThreads;
-  // encoder shared memory per warp: the row (128-byte aligned) and a stash of one outlier per
-  // 32 elements (rows with more take a slower path)
-  p->enc_row_stride = (p->row_bytes + 127u) & ~127u;
-  p->enc_stash_cap = (p->units * 4u + 127u) / 128u * 32u;
-  p->enc_warp_stride = p->enc_row_stride + p->enc_stash_cap * 4u;
+  // encoder: one thread per 32-element group, two for rows longer than kEncMaxThreads groups
+  p->enc_upt = p->units > static_cast<uint32_t>(kEncMaxThreads) ? 2 : 1;
+  p->enc_threads = static_cast<int>(((p->units + p->enc_upt - 1) / p->enc_upt + 31u) / 32u * 32u);
   p->dec_smem = decode_smem_bytes(p->row_bytes);
   const unsigned long long desc = T > 0 ? T : 1;
-  p->workspace_bytes = static_cast<size_t>(align16(sizeof(WsControl) + 12ull * desc));
+  p->workspace_bytes = static_cast<size_t>(align16(sizeof(WsControl) + 16ull * desc));
 
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) {
@@ -145,17 +142,8 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   int prev_dev = 0;
   cudaGetDevice(&prev_dev);
   bool ok = cudaSetDevice(device) == cudaSuccess;
-  int sms = 0, dec_blocks = 0, smem_optin = 0;
+  int sms = 0, dec_blocks = 0;
   ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess;
-  ok = ok && cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) == cudaSuccess;
-  if (ok) {
-    // one encoder CTA per SM, as many row slots as fit beside the kernel's static shared memory
-    long long w = (static_cast<long long>(smem_optin) - 1024) / static_cast<long long>(p->enc_warp_stride);
-    if (w > kEncMaxWarps) w = kEncMaxWarps;
-    p->enc_warps = static_cast<int>(w);
-    ok = w >= 1;
-  }
-  ok = ok && encode_kernel_attrs(dtype == TSQ_BF16, static_cast<size_t>(p->enc_warps) * p->enc_warp_stride) == cudaSuccess;
   ok = ok && decode_kernel_attrs(dtype == TSQ_BF16, p->threads, p->dec_smem, &dec_blocks) == cudaSuccess;
   cudaSetDevice(prev_dev);
   if (!ok || dec_blocks < 1 || sms < 1) {
@@ -209,9 +197,7 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
   p.x = static_cast<const uint16_t*>(x_dev);
   p.blob = static_cast<unsigned char*>(blob_dev);
   p.ws = static_cast<WsControl*>(ws_dev);
-  const unsigned long long desc = plan->max_tokens > 0 ? plan->max_tokens : 1;
   p.desc = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(ws_dev) + sizeof(WsControl));
-  p.prefix_outl = reinterpret_cast<uint32_t*>(p.desc + desc);
   p.lay = L;
   p.tokens = static_cast<uint32_t>(tokens);
   p.hidden = plan->hidden;
@@ -221,24 +207,14 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
   p.n_bits = plan->n_bits;
   for (int i = 0; i < 8; ++i) p.bits[i] = plan->bits[i];
   p.s_max = plan->s_max;
-  p.row_bytes = plan->row_bytes;
-  p.row_stride = plan->enc_row_stride;
-  p.warp_stride = plan->enc_warp_stride;
-  p.stash_cap = plan->enc_stash_cap;
-  p.bulk_store = (plan->units % 4u == 0u) ? 1u : 0u;
+  p.vec_store = (plan->units % 4u == 0u) ? 1u : 0u;
   p.dtype = static_cast<uint32_t>(plan->dtype);
   p.tau = plan->tau;
   p.delta = plan->delta;
 
-  // rows are spread over the SMs first, then over the warps of each CTA
-  int grid = tokens < plan->sms ? static_cast<int>(tokens) : plan->sms;
-  if (grid < 1) grid = 1;
-  long long active = (tokens + grid - 1) / grid;
-  if (active > plan->enc_warps) active = plan->enc_warps;
-  if (active < 1) active = 1;
-  p.active_warps = static_cast<uint32_t>(active);
-  const cudaError_t e = launch_encode(p, grid, plan->enc_warps * 32, static_cast<size_t>(plan->enc_warps) * plan->enc_warp_stride,
-                                      static_cast<cudaStream_t>(cuda_stream));
+  // one CTA per row; a call without rows still launches one CTA, which writes the header
+  const int grid = tokens > 0 ? static_cast<int>(tokens) : 1;
+  const cudaError_t e = launch_encode(p, grid, plan->enc_threads, plan->enc_upt, static_cast<cudaStream_t>(cuda_stream));
   g_launches.fetch_add(1);
   return e == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
 }

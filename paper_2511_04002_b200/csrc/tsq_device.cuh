@@ -104,7 +104,7 @@ struct Elem<false> {  // IEEE binary16
   // two non-negative binary32 values -> packed 16-bit, round-to-nearest-even
   static __device__ __forceinline__ uint32_t pack_rn(float lo, float hi) { return bits(__floats2half2_rn(lo, hi)); }
   // largest pattern whose value is <= f (f >= 0)
-  static __device__ __forceinline__ uint32_t pattern_rd(float f) { return __half_as_ushort(__float2half_rd(f)); }
+  static __device__ __forceinline__ uint32_t pattern_rd(float f) { return __half_as_ushort(__float2half_rz(f)); }
 };
 
 template <>
@@ -119,9 +119,7 @@ struct Elem<true> {  // bfloat16
   static __device__ __forceinline__ float hi_f32(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
   static __device__ __forceinline__ float pattern_f32(uint32_t p) { return __uint_as_float(p << 16); }
   static __device__ __forceinline__ uint32_t pack_rn(float lo, float hi) { return bits(__floats2bfloat162_rn(lo, hi)); }
-  static __device__ __forceinline__ uint32_t pattern_rd(float f) {
-    return __bfloat16_as_ushort(__float2bfloat16_rd(f));
-  }
+  static __device__ __forceinline__ uint32_t pattern_rd(float f) { return __float_as_uint(f) >> 16; }
 };
 
 // ---- 8 x 32 bit-matrix transpose -------------------------------------------------------------------

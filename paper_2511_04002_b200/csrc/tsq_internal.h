@@ -14,7 +14,7 @@ constexpr uint32_t kMagic = 0x31515354u;  // 'T','S','Q','1'
 constexpr uint32_t kVersion = 1u;
 constexpr int kMaxCand = 7;
 constexpr int kMaxThreads = 256;          // decoder: threads per CTA, one 32-element unit per thread per pass
-constexpr int kEncMaxWarps = 16;          // encoder: warps per CTA, one row in flight per warp
+constexpr int kEncMaxThreads = 1024;      // encoder: one CTA per row, one or two 32-element groups per thread
 
 struct BlobHeader {
   uint32_t magic, version, dtype, hidden, tokens, n_bits;
@@ -53,9 +53,9 @@ __host__ __device__ inline BlobLayout make_layout(uint32_t hidden, unsigned long
   return L;
 }
 
-// Workspace: a 64-byte control block, one 64-bit descriptor per token and one 32-bit outlier
-// prefix per token.  A descriptor is (tag << 32) | value with tag = generation * 4 + flag; stale
-// generations read as "not yet published", so the arrays never need clearing between calls.
+// Workspace: a 64-byte control block and two adjacent 64-bit descriptors per token (plane words,
+// outliers).  A descriptor is (tag << 32) | value with tag = generation * 4 + flag; stale
+// generations read as "not yet published", so the array never needs clearing between calls.
 struct WsControl {
   uint32_t gen;          // generation of the last finished encode
   uint32_t ticket;       // next tile to hand out (self-resetting)
@@ -63,7 +63,7 @@ struct WsControl {
   uint32_t err;          // first error of the running encode
   uint32_t enc_status;   // first encode error since init (sticky)
   uint32_t dec_status;   // first decode error since init (sticky)
-  uint32_t desc_capacity;  // descriptors per array (set by init)
+  uint32_t desc_capacity;  // tiles the descriptor array holds (set by init)
   uint32_t pad[9];
 };
 static_assert(sizeof(WsControl) == 64, "control block is 64 bytes");
@@ -75,19 +75,14 @@ struct EncodeParams {
   const uint16_t* x;
   unsigned char* blob;
   WsControl* ws;
-  unsigned long long* desc;                  // [max_tokens] tile descriptors
-  uint32_t* prefix_outl;                     // [max_tokens] inclusive outlier prefixes
+  unsigned long long* desc;                  // [2 * max_tokens] tile descriptors
   BlobLayout lay;
   uint32_t tokens, hidden, units, chunks;   // units = ceil(H/32), chunks = H/8
   uint32_t thr16;                            // smallest non-negative 16-bit pattern with value >= tau
   int32_t n_bits;
   int32_t bits[8];
   int32_t s_max;                             // floor(delta * H), clamped to [-1, INT32_MAX]
-  uint32_t row_bytes;                        // bytes of one input row
-  uint32_t row_stride, warp_stride;          // shared memory per warp: row slot, and row slot + outlier stash
-  uint32_t stash_cap;                        // entries of the outlier stash
-  uint32_t bulk_store;                       // 1: every token's plane words are a multiple of 16 bytes
-  uint32_t active_warps;                     // warps of each CTA that take rows
+  uint32_t vec_store;                        // 1: every token's plane words start on a 16-byte boundary
   uint32_t dtype;
   float tau, delta;
 };
@@ -102,9 +97,8 @@ struct DecodeParams {
   unsigned long long blob_bytes;
 };
 
-cudaError_t launch_encode(const EncodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
+cudaError_t launch_encode(const EncodeParams& p, int grid, int threads, int groups_per_thread, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
-cudaError_t encode_kernel_attrs(bool bf16, size_t smem);
 cudaError_t decode_kernel_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm);
 size_t decode_smem_bytes(uint32_t row_bytes);
 
