@@ -121,6 +121,30 @@ tsq_status_t tsq_encode(const tsq_plan_t *plan, const void *x_dev, int64_t token
                         size_t blob_bytes, void *ws_dev, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The same encode as tsq_encode, for callers that cannot give it a workspace.  (The paper has no
+ * counterpart: this is a convenience of the library.)  Some hosts of this codec are not allowed to
+ * allocate device memory where they call it: code running inside a region that forbids allocation
+ * (a latency-critical serving loop with a frozen memory pool, a plug-in whose embedding runtime owns
+ * all device memory, a thread that must never take the allocator's lock).  For them the look-back
+ * scratch lives in a fixed array inside the library image instead of in a caller-allocated workspace;
+ * x_dev and blob_dev are still the caller's.
+ *   - Limit: the plan's max_tokens must be <= 16384 (the array is 256 KiB + 256 B per device, held
+ *     by every device that loads the library until the process exits); larger plans are refused with
+ *     TSQ_ERR_UNSUPPORTED before anything is enqueued.
+ *   - The call allocates and frees nothing.  The first call on a device looks up the array's device
+ *     address (a one-time host-side query with that device made current for a moment); make that
+ *     first call before any stream capture begins.
+ *   - Each call first clears the part of the array it uses, on `cuda_stream`, then encodes.  All calls
+ *     on a device share the one array: two calls whose work may overlap on the GPU (different
+ *     streams, no ordering between them) race on it and corrupt each other's placement.  Order them
+ *     on one stream or with events.
+ *   - Asynchronous conditions are reported in the blob header only (read them with tsq_blob_info).
+ * Output, arguments and errors are otherwise those of tsq_encode.
+ */
+tsq_status_t tsq_encode_noalloc(const tsq_plan_t *plan, const void *x_dev, int64_t tokens, void *blob_dev,
+                                size_t blob_bytes, void *cuda_stream);
+
+/*
  * Decode blob (DEVICE) into y (DEVICE, [tokens x hidden]): Eq. "dequnt".  The kernel validates the
  * header against the plan and `tokens`, and every per-token field against the blob's capacities,
  * before using it; on a mismatch it writes nothing for that blob/row and records

@@ -16,7 +16,8 @@ F16, BF16 = 0, 1
 STATUS = {0: "TSQ_OK", 1: "TSQ_ERR_INVALID_ARG", 2: "TSQ_ERR_UNSUPPORTED", 3: "TSQ_ERR_BUFFER_TOO_SMALL",
           4: "TSQ_ERR_CUDA", 5: "TSQ_ERR_CORRUPT_BLOB", 6: "TSQ_ERR_OUTLIER_OVERFLOW", 7: "TSQ_ERR_TIMEOUT"}
 
-EXPORTS = ["tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_encode", "tsq_decode", "tsq_blob_info",
+EXPORTS = ["tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_encode", "tsq_encode_noalloc", "tsq_decode",
+           "tsq_blob_info",
            "tsq_workspace_status", "tsq_encode_host", "tsq_decode_host", "tsq_kernel_launch_count",
            "tsq_plan_destroy", "tsq_status_string"]
 
@@ -54,6 +55,8 @@ def lib() -> C.CDLL:
     L.tsq_plan_sizes.argtypes = [vp, i64, C.POINTER(_Sizes)]
     L.tsq_workspace_init.argtypes = [vp, vp, sz, vp]
     L.tsq_encode.argtypes = [vp, vp, i64, vp, sz, vp, sz, vp]
+    L.tsq_encode_noalloc.argtypes = [vp, vp, i64, vp, sz, vp]
+    L.tsq_encode_noalloc.restype = C.c_int
     L.tsq_decode.argtypes = [vp, vp, sz, i64, vp, vp, sz, vp]
     L.tsq_blob_info.argtypes = [vp, C.POINTER(_Info), vp]
     L.tsq_workspace_status.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), vp]
@@ -142,6 +145,12 @@ class Plan:
         assert x.is_cuda and x.is_contiguous() and x.dtype == self.dtype and x.dim() == 2 and x.shape[1] == self.hidden
         _check(lib().tsq_encode(self._h, x.data_ptr(), x.shape[0], blob.data_ptr(), blob.numel(), ws.data_ptr(),
                                 ws.numel(), _stream(stream)), "tsq_encode")
+
+    def encode_noalloc(self, x: torch.Tensor, blob: torch.Tensor, stream=None) -> None:
+        """tsq_encode_noalloc: encode with the library's built-in scratch array instead of a workspace."""
+        assert x.is_cuda and x.is_contiguous() and x.dtype == self.dtype and x.dim() == 2 and x.shape[1] == self.hidden
+        _check(lib().tsq_encode_noalloc(self._h, x.data_ptr(), x.shape[0], blob.data_ptr(), blob.numel(),
+                                        _stream(stream)), "tsq_encode_noalloc")
 
     def decode(self, blob: torch.Tensor, tokens: int, y: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
         assert y.is_cuda and y.is_contiguous() and y.dtype == self.dtype and tuple(y.shape) == (tokens, self.hidden)

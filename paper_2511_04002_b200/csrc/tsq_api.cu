@@ -3,6 +3,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "tsq_internal.h"
@@ -45,6 +46,38 @@ uint32_t threshold_pattern(tsq_dtype_t dtype, float tau) {
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Scratch of tsq_encode_noalloc: a workspace that lives in the library image instead of in memory the
+// caller allocates.  Every device that loads the library holds its own copy until the process exits.
+constexpr unsigned long long kStaticMaxTokens = 16384;
+constexpr size_t kStaticWsBytes = (sizeof(WsControl) + 16ull * kStaticMaxTokens + 255ull) & ~255ull;
+static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
+
+// In host code `g_static_ws` is only a handle for the runtime, not an address a kernel may use: the
+// device address is asked for once per device, with that device current, and kept here.
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};
+
+cudaError_t static_workspace(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[device]) {
+    int prev = 0;
+    cudaError_t e = cudaGetDevice(&prev);
+    if (e != cudaSuccess) return e;
+    e = cudaSetDevice(device);
+    if (e != cudaSuccess) return e;
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_ws);
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) return e;
+    if (!ptr) return cudaErrorInvalidSymbol;
+    g_static_ptr[device] = ptr;
+  }
+  *out = g_static_ptr[device];
+  return cudaSuccess;
+}
 
 __global__ void workspace_init_kernel(WsControl* ws, uint32_t desc_capacity) { ws->desc_capacity = desc_capacity; }
 
@@ -246,6 +279,23 @@ tsq_status_t tsq_decode(const tsq_plan_t* plan, const void* blob_dev, size_t blo
                                       static_cast<cudaStream_t>(cuda_stream));
   g_launches.fetch_add(1);
   return e == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
+}
+
+tsq_status_t tsq_encode_noalloc(const tsq_plan_t* plan, const void* x_dev, int64_t tokens, void* blob_dev,
+                                size_t blob_bytes, void* cuda_stream) {
+  if (!plan) return TSQ_ERR_INVALID_ARG;
+  if (plan->max_tokens > kStaticMaxTokens || plan->workspace_bytes > kStaticWsBytes) return TSQ_ERR_UNSUPPORTED;
+  void* ws = nullptr;
+  if (static_workspace(plan->device, &ws) != cudaSuccess) {
+    cudaGetLastError();
+    return TSQ_ERR_CUDA;
+  }
+  // the array keeps whatever the last call left (including an unfinished call's tickets): start clean
+  if (cudaMemsetAsync(ws, 0, plan->workspace_bytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return TSQ_ERR_CUDA;
+  }
+  return tsq_encode(plan, x_dev, tokens, blob_dev, blob_bytes, ws, kStaticWsBytes, cuda_stream);
 }
 
 static unsigned long long payload_of(unsigned long long tokens, unsigned long long words, unsigned long long outliers) {
