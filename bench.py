@@ -34,7 +34,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from paper_2511_04002_b200 import synth
+from paper_2511_04002_b200 import shard, synth
 
 METRIC = "TS+TAB-Q encode+decode throughput (algorithmic bytes: 16-bit tensor + payload, both directions)"
 UNIT = "GB/s"
@@ -344,13 +344,7 @@ def run_tsq(args, w):
     for s in sets:
         assert plan.workspace_status(s.ws) == (0, 0), "codec reported an error in the timed region"
 
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-        b = torch.tensor([float(bytes_done), float(launches)], dtype=torch.float64, device="cuda")
-        dist.all_reduce(b, op=dist.ReduceOp.SUM)
-        bytes_done, launches = float(b[0].item()), int(b[1].item())
+    total_ms, bytes_done, launches = shard.reduce_job(total_ms, bytes_done, launches, "cuda")
 
     # ---- end to end: host tensors in and out, copies inside the timed region (every rank, in parallel)
     e2e = None
@@ -373,10 +367,7 @@ def run_tsq(args, w):
         torch.cuda.synchronize()
         barrier()
         e2e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms, _, _ = shard.reduce_job(e2e_ms, 0, 0, "cuda")
         e2e = {"value": world * n_e2e * 2 * (x_bytes + payload) / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": x_bytes + payload, "d2h_bytes_per_step": payload + x_bytes,
                "steps": n_e2e, "ms_per_step": e2e_ms / n_e2e,

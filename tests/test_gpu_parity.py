@@ -259,3 +259,49 @@ def test_run_to_run_determinism_and_host_calls():
     y_dev = torch.empty_like(x, device="cuda")
     plan.decode_host(blob_host, T, y_host, blob, y_dev, ws)
     assert np.array_equal(synth.raw_u16(y_host), R.decode(a))
+
+
+# ------------------------------------------------------------------ full size, as the benchmark launches it
+
+def test_c4_full_size_sampled_rows_and_invariants():
+    """The benchmark's workload at its full size (8192 x 8192 bf16), same plan and launch shape.
+    The oracle encodes sampled rows one by one; the rest is checked through properties that hold at any size."""
+    w = synth.c4_70b_prefill()
+    x = synth.make(w)
+    T, H = x.shape
+    plan = B.Plan(x.dtype, H, T, w.tau, list(w.bits), w.delta)
+    blob, ws = plan.alloc(T)
+    xd = x.cuda()
+    plan.encode(xd, blob, ws)
+    y = torch.empty_like(xd)
+    plan.decode(blob, T, y, ws)
+    torch.cuda.synchronize()
+    assert plan.workspace_status(ws) == (0, 0)
+    host = blob.cpu().numpy()
+    hdr, sec = R.header(host), R.sections(host)
+    wpp = H // 32
+    raw = synth.raw_u16(x)
+    # placement: plain prefix sums, outlier counts equal an independent count of |x| >= tau (NaN/Inf included)
+    assert np.array_equal(sec["word_off"], np.concatenate([[0], np.cumsum(sec["bits"].astype(np.int64) * wpp)]))
+    out = ~(x.float().abs() < w.tau)
+    assert np.array_equal(np.diff(sec["out_ptr"].astype(np.int64)), out.sum(dim=1).numpy())
+    assert hdr["total_words"] == int(sec["word_off"][-1]) and hdr["total_outliers"] == int(sec["out_ptr"][-1])
+    # CSR: ascending columns per row, original patterns
+    rows_of = np.repeat(np.arange(T), np.diff(sec["out_ptr"].astype(np.int64)))
+    cols = (sec["outl"] >> 16).astype(np.int64)
+    assert np.array_equal(raw[rows_of, cols], (sec["outl"] & 0xffff).astype(np.uint16))
+    same_row = rows_of[1:] == rows_of[:-1]
+    assert np.all(cols[1:][same_row] > cols[:-1][same_row])
+    # outliers come back bit-exactly in the reconstruction
+    y_raw = synth.raw_u16(y.cpu())
+    assert np.array_equal(y_raw[out.numpy()], raw[out.numpy()])
+    # sampled rows against the oracle, element by element: fields, plane words, reconstruction
+    rng = np.random.default_rng(0)
+    for t in sorted(set([0, 1, T - 1] + rng.integers(0, T, 61).tolist())):
+        ref = R.encode(raw[t:t + 1], R.BF16, w.tau, list(w.bits), w.delta)
+        rs = R.sections(ref)
+        assert sec["bits"][t] == rs["bits"][0] and sec["zp"][t] == rs["zp"][0]
+        assert sec["scale"][t:t + 1].view(np.uint32)[0] == rs["scale"].view(np.uint32)[0]
+        assert np.array_equal(sec["words"][sec["word_off"][t]:sec["word_off"][t + 1]], rs["words"])
+        assert np.array_equal(sec["outl"][sec["out_ptr"][t]:sec["out_ptr"][t + 1]], rs["outl"])
+        assert np.array_equal(y_raw[t], R.decode(ref)[0])
