@@ -96,7 +96,11 @@ struct tsq_plan {
   int32_t s_max;
   uint32_t thr16;
   int threads;                      // decoder CTA size
-  int enc_threads, enc_upt;         // encoder CTA size and 32-element groups per thread
+  int enc_threads, enc_upt;         // row-at-a-time encoder: CTA size and 32-element groups per thread
+  // pipelined encoder: 0 CTAs per SM when the row does not fit its shared memory
+  int pipe_threads, pipe_ctas_per_sm;
+  uint32_t pipe_compute, pipe_park, pipe_planes, pipe_csr_cap;
+  size_t pipe_smem;
   int sms;
   size_t dec_smem;
   size_t workspace_bytes;
@@ -178,6 +182,23 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   int sms = 0, dec_blocks = 0;
   ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess;
   ok = ok && decode_kernel_attrs(dtype == TSQ_BF16, p->threads, p->dec_smem, &dec_blocks) == cudaSuccess;
+  {
+    // pipelined encoder: three parked rows, four rows of planes and of CSR entries per CTA
+    int smem_optin = 0;
+    ok = ok && cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) == cudaSuccess;
+    p->pipe_compute = (p->units + 31u) / 32u * 32u;
+    p->pipe_threads = static_cast<int>(p->pipe_compute) + 64;
+    p->pipe_park = p->pipe_compute * 64u;
+    p->pipe_planes = (static_cast<uint32_t>(p->bmax) * p->units * 4u + 127u) & ~127u;
+    p->pipe_csr_cap = p->units < 64u ? 64u : p->units;
+    p->pipe_smem = 3u * static_cast<size_t>(p->pipe_park) + 4u * static_cast<size_t>(p->pipe_planes) + 16u * static_cast<size_t>(p->pipe_csr_cap);
+    p->pipe_ctas_per_sm = 0;
+    if (ok && p->pipe_threads <= 1024 && p->pipe_smem + 8192 <= static_cast<size_t>(smem_optin)) {
+      int blocks = 0;
+      ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_threads, p->pipe_smem, &blocks) == cudaSuccess;
+      p->pipe_ctas_per_sm = blocks;
+    }
+  }
   cudaSetDevice(prev_dev);
   if (!ok || dec_blocks < 1 || sms < 1) {
     cudaGetLastError();
@@ -245,9 +266,22 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
   p.tau = plan->tau;
   p.delta = plan->delta;
 
-  // one CTA per row; a call without rows still launches one CTA, which writes the header
-  const int grid = tokens > 0 ? static_cast<int>(tokens) : 1;
-  const cudaError_t e = launch_encode(p, grid, plan->enc_threads, plan->enc_upt, static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e;
+  if (plan->pipe_ctas_per_sm > 0 && tokens > 2 * static_cast<int64_t>(plan->sms)) {
+    // many rows: persistent CTAs that overlap the stages of consecutive rows
+    p.compute_threads = plan->pipe_compute;
+    p.park_stride = plan->pipe_park;
+    p.planes_stride = plan->pipe_planes;
+    p.csr_cap = plan->pipe_csr_cap;
+    const long long resident = static_cast<long long>(plan->sms) * plan->pipe_ctas_per_sm;
+    const int grid = static_cast<int>(tokens < resident ? tokens : resident);
+    e = launch_encode_pipe(p, grid, plan->pipe_threads, plan->pipe_smem, static_cast<cudaStream_t>(cuda_stream));
+  } else {
+    // few rows (or rows too long for the pipeline): one CTA per row; a call without rows still launches
+    // one CTA, which writes the header
+    const int grid = tokens > 0 ? static_cast<int>(tokens) : 1;
+    e = launch_encode_rows(p, grid, plan->enc_threads, plan->enc_upt, static_cast<cudaStream_t>(cuda_stream));
+  }
   g_launches.fetch_add(1);
   return e == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
 }

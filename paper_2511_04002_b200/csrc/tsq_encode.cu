@@ -1,18 +1,28 @@
-// tsq encode kernel: threshold splitting (Eq. "ts") + token-wise TAB-Q (Algorithm 1 on AIQ,
+// tsq encode kernels: threshold splitting (Eq. "ts") + token-wise TAB-Q (Algorithm 1 on AIQ,
 // Eq. "Proposed") + bit-plane packing + CSR emission, fused into one kernel.
 //
-// One CTA encodes one token row, one thread per group of 32 elements (two groups per thread for
-// rows longer than 32768).  A thread loads its group's 64 bytes straight into registers and the
-// row never leaves them: the input is read from HBM exactly once, there is no staging copy, and
-// every pass of the method is straight-line register arithmetic:
+// One CTA encodes one token row at a time, one thread per group of 32 elements.  A thread loads its
+// group's 64 bytes straight into registers, so the input is read from HBM exactly once.  The passes:
 //   A  threshold split: outlier bitmap, outlier slots set to +0 (what T_below holds there), and
 //      the row's min / max of the inlier magnitudes (CTA reduction);
 //   B  Algorithm 1: AIQ codes at the top level and at each lower candidate, distortion sums
 //      (CTA reduction, one candidate at a time, stopping at the first failure);
 //   C  codes at the chosen level -> bytes (code | sign << 7) -> 8 x 32 bit transpose -> the
-//      group's b* plane words, stored as one contiguous run per thread.
-// The scalar work between the passes (scales, zero-points, the check described below, the
-// placement) is done by warp 0 alone; the other CTAs resident on the SM fill those gaps.
+//      group's b* plane words, one contiguous run per thread.
+// Between the passes sits scalar work per row (the AIQ parameters of every candidate: a few
+// divisions) and the placement of the row's output, which has to wait for every earlier row.
+//
+// Two kernels share the passes:
+//   encode_rows_kernel  one CTA per row, everything in order; used for few rows (lowest latency per
+//                       call) and for rows too long for the pipeline's shared memory.
+//   encode_pipe_kernel  persistent CTAs that keep several rows in different stages at once, so that
+//                       the vector passes never wait for the scalar work or for the placement:
+//                       the compute warps run pass A of row n (parking the thresholded row in
+//                       shared memory), then passes B and C of row n - 1 from its parked copy; a
+//                       "levels" warp turns row n's min / max into AIQ parameters meanwhile; a
+//                       "placement" warp resolves the offsets of rows packed earlier, ships their
+//                       planes with one bulk asynchronous store each and writes their CSR entries.
+//                       The next row's global loads are issued before passes B and C start.
 //
 // The binding resource is the integer / logic pipe, which issues at half the rate of the FMA pipe:
 // the passes work on two 16-bit elements per 32-bit register wherever they can, and shifts and
@@ -20,27 +30,20 @@
 //
 // Variable-length placement: where a token's planes and CSR entries start is an exclusive prefix
 // sum over all earlier tokens.  It is resolved with a decoupled look-back over per-token
-// descriptors in the workspace.  Rows are numbered by an atomic ticket taken when a CTA starts,
-// so a row only ever waits for rows whose CTAs are already running.  A row publishes its own
-// sizes right after pass B and looks back only after pass C, so that the wait for slower
-// predecessors overlaps its own packing.  A look-back step reads 256 descriptors at once (eight
+// descriptors in the workspace.  Rows are numbered by an atomic ticket taken by a running CTA,
+// so a row only ever waits for rows whose CTAs are already running, and a row publishes its own
+// sizes before it waits for anything.  A look-back step reads 256 descriptor pairs at once (eight
 // independent loads per lane).  Every wait is bounded and fails into a status word.
 //
 // Arithmetic contract: the codes equal  clamp(rint(m / s) - zp, 0, Qmax)  with the IEEE binary32
-// quotient m / s.  Three evaluations of it exist, chosen per row:
-//   kFast     rint(m * r) with r = fl(1/s), one FMA against 2^23.  It can differ from the
-//             contract only when m / s lies within a relative 2^-22 of a rounding boundary k + 1/2
-//             (exact ties included: 16-bit inputs make m / s land exactly on k + 1/2 quite often).
-//             16-bit values are at least 2^-11 apart, so for each boundary only its two
-//             neighbouring 16-bit values can be affected; those are examined per row, a cheap
-//             distance test first and the true division for the few that fail it.
-//   kRefined  for a row where any of them really disagrees: the correctly rounded quotient from
-//             q0 = fl(m * r), the exact residual m - q0 * s (one FMA) and q = fl(q0 + residual * r)
-//             (the classical FMA division step, exact when r is the correctly rounded reciprocal
-//             and nothing over- or underflows), then the same 2^23 rounding.
-//   kDivide   the division instruction itself, for rows whose scale is so large or so small that
-//             the intermediate products of the other two could leave the normal range, or whose
-//             zero-point does not fit the packed 16-bit integer steps of the other two.
+// quotient m / s.  The quotient is formed without the division instruction: r = fl(1 / s) once per
+// row and level, then per element q0 = fl(m * r), the exact residual m - q0 * s (one FMA) and
+// q = fl(q0 + residual * r).  This is the classical FMA division step: with a correctly rounded
+// reciprocal and no over- or underflow, q is the correctly rounded quotient.  (A single
+// fl(m * r) is not enough: 16-bit inputs put m / s on or next to a rounding boundary k + 1/2 in
+// almost every row, and there the two can round differently.)  rint is one addition of 2^23.  Rows
+// whose scale is so large or so small that an intermediate product could leave the normal range,
+// or whose zero-point does not fit the packed 16-bit integer steps, use the division instruction.
 
 #include "tsq_device.cuh"
 #include "tsq_internal.h"
@@ -51,7 +54,8 @@ namespace {
 constexpr float kRoundMagic = 8388608.0f;  // 2^23: adding it to 0 <= y < 2^23 rounds y to an integer, ties to even
 constexpr uint32_t kRoundMagicHi = 0x4B00u;  // upper 16 bits of the pattern of 2^23
 constexpr uint32_t kLookbackPollLimit = 1u << 20;
-constexpr int kLookbackDepth = 8;  // descriptors each lane reads per look-back step
+constexpr uint32_t kHandshakePollLimit = 1u << 22;
+constexpr int kLookbackDepth = 8;  // descriptor pairs each lane reads per look-back step
 
 // AIQ parameters of one candidate level for one row (Eq. "Proposed").
 struct Level {
@@ -61,10 +65,8 @@ struct Level {
   int qmax;      // 2^(b-1) - 1
   uint32_t nz2;  // -zp in the low half, -zp - kRoundMagicHi in the high half (see codes2)
   uint32_t qm2;  // qmax in both 16-bit halves
-  bool fast;     // scale and zero-point in the range where the FMA paths are provably safe
+  int packed;    // scale and zero-point in the range where the FMA quotient and the packed steps are safe
 };
-
-enum Mode : int { kFast = 0, kRefined = 1, kDivide = 2 };
 
 __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
   Level c;
@@ -76,87 +78,27 @@ __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
   c.nz2 = (static_cast<uint32_t>(-c.zp) & 0xffffu) | (static_cast<uint32_t>(-c.zp - static_cast<int>(kRoundMagicHi)) << 16);
   c.qm2 = static_cast<uint32_t>(c.qmax) * 0x10001u;
   // rint(m / s) <= zp + qmax + 1 must stay a small positive 16-bit integer for the packed steps
-  c.fast = (c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && (c.zp < 12000);
+  c.packed = ((c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && (c.zp < 12000)) ? 1 : 0;
   return c;
 }
 
-// Code of one magnitude (scalar form: boundary checks only).
-template <int MODE>
-__device__ __forceinline__ int code_of(float m, const Level& c) {
-  int k;
-  if (MODE == kFast) {
-    k = (__float_as_int(fmaf(m, c.r, kRoundMagic)) & 0xffff) - c.zp;
-  } else {
-    k = __float2int_rn(__fdiv_rn(m, c.s)) - c.zp;
-  }
-  return __vimin_s32_relu(k, c.qmax);  // clamp to [0, qmax]
-}
-
 // Codes of the two elements of a 16-bit pair (sign bits ignored), as two 16-bit integers.
-template <bool BF16, int MODE>
+template <bool BF16, bool DIVIDE>
 __device__ __forceinline__ uint32_t codes2(uint32_t x, const Level& c) {
   using E = Elem<BF16>;
   const float lo = fabsf(E::lo_f32(x)), hi = fabsf(E::hi_f32(x));
-  if (MODE == kDivide) {
+  if (DIVIDE) {
     const int klo = __vimin_s32_relu(__float2int_rn(__fdiv_rn(lo, c.s)) - c.zp, c.qmax);
     const int khi = __vimin_s32_relu(__float2int_rn(__fdiv_rn(hi, c.s)) - c.zp, c.qmax);
     return static_cast<uint32_t>(klo) | (static_cast<uint32_t>(khi) << 16);
   }
-  float tlo, thi;
-  if (MODE == kFast) {
-    tlo = fmaf(lo, c.r, kRoundMagic);
-    thi = fmaf(hi, c.r, kRoundMagic);
-  } else {
-    const float q0 = __fmul_rn(lo, c.r), q1 = __fmul_rn(hi, c.r);
-    tlo = __fadd_rn(fmaf(fmaf(-q0, c.s, lo), c.r, q0), kRoundMagic);  // fl(lo / s), then to an integer
-    thi = __fadd_rn(fmaf(fmaf(-q1, c.s, hi), c.r, q1), kRoundMagic);
-  }
-  // pattern of 2^23 + k = 0x4B000000 + k.  thi * 2^16 + tlo (mod 2^32) = (0x4B00 + k_lo's carry-free
-  // neighbour k_hi) << 16 | k_lo; the constant in the high half is taken off together with zp.
+  const float q0 = __fmul_rn(lo, c.r), q1 = __fmul_rn(hi, c.r);
+  const float tlo = __fadd_rn(fmaf(fmaf(-q0, c.s, lo), c.r, q0), kRoundMagic);  // fl(lo / s), then to an integer
+  const float thi = __fadd_rn(fmaf(fmaf(-q1, c.s, hi), c.r, q1), kRoundMagic);
+  // pattern of 2^23 + k = 0x4B000000 + k, so thi * 2^16 + tlo (mod 2^32) = (0x4B00 + k_hi) << 16 | k_lo;
+  // the constant in the high half is taken off together with zp.
   const uint32_t k2 = __float_as_uint(thi) * 65536u + __float_as_uint(tlo);
   return __viaddmin_s16x2_relu(k2, c.nz2, c.qm2);  // clamp(k - zp, 0, qmax) in both halves
-}
-
-// Does the fast path disagree with the true division for a 16-bit value next to rounding
-// boundary (zp + j - 1/2) * s ?  Only values inside [pmin, pmax] can occur in the row.
-template <bool BF16>
-__device__ __forceinline__ bool boundary_disagrees(const Level& c, int j, uint32_t pmin, uint32_t pmax) {
-  using E = Elem<BF16>;
-  const float h = static_cast<float>(c.zp + j) - 0.5f;
-  if (!(h > 0.0f)) return false;
-  const float centre = __fmul_rn(h, c.s);
-  const uint32_t plo = E::pattern_rd(centre);
-  const float margin = __fmul_rn(h, 0x1p-21f);
-  bool bad = false;
-#pragma unroll
-  for (uint32_t d = 0; d < 2; ++d) {
-    const uint32_t pat = plo + d;
-    if (pat >= pmin && pat <= pmax) {
-      const float m = E::pattern_f32(pat);
-      // |m * r - h| > h * 2^-21 puts m / s more than h * 2^-22 away from the boundary: both paths agree
-      if (fabsf(__fsub_rn(__fmul_rn(m, c.r), h)) <= margin) bad |= code_of<kFast>(m, c) != code_of<kDivide>(m, c);
-    }
-  }
-  return bad;
-}
-
-// Examine every rounding boundary of every candidate level, one boundary per thread at a time
-// (the levels' boundaries are numbered end to end, the top level first).
-template <bool BF16>
-__device__ __forceinline__ bool any_boundary_disagrees(const Level* lv, int n_levels, uint32_t pmin, uint32_t pmax,
-                                                       uint32_t tid, uint32_t nthreads) {
-  int total = 0;
-  for (int i = 0; i < n_levels; ++i) total += lv[i].qmax + 2;
-  bool bad = false;
-  for (int t = static_cast<int>(tid); t < total; t += static_cast<int>(nthreads)) {
-    int i = n_levels - 1, j = t;
-    while (j >= lv[i].qmax + 2) {
-      j -= lv[i].qmax + 2;
-      --i;
-    }
-    bad |= boundary_disagrees<BF16>(lv[i], j, pmin, pmax);
-  }
-  return bad;
 }
 
 __device__ __forceinline__ uint32_t max_s16x2(uint32_t a, uint32_t b) {
@@ -202,36 +144,127 @@ __device__ __forceinline__ uint32_t split_group(uint32_t (&x)[16], uint32_t nval
 }
 
 // Pass B on one group: sum |(q0 >> sh) - q| over its 32 elements (Algorithm 1's distortion numerator).
-template <bool BF16, int MODE>
+template <bool BF16, bool DIVIDE>
 __device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], const Level& top, const Level& low,
                                                      int sh) {
   const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
   uint32_t S2 = 0;  // two 16-bit partial sums: at most 16 * 127 each
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    const uint32_t a = (codes2<BF16, MODE>(x[i], top) >> sh) & shmask;
-    const uint32_t q = codes2<BF16, MODE>(x[i], low);
+    const uint32_t a = (codes2<BF16, DIVIDE>(x[i], top) >> sh) & shmask;
+    const uint32_t q = codes2<BF16, DIVIDE>(x[i], low);
     S2 += max_s16x2(a, q) - min_s16x2(a, q);
   }
   return (S2 & 0xffffu) + (S2 >> 16);
 }
 
+// Pass B for the first lower candidate, keeping what pass C needs if that candidate fails: on return
+// b2[i] holds the top-level bytes (code | sign << 7) of pair i, low element in byte 0, high in byte 2.
+template <bool BF16, bool DIVIDE>
+__device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], const Level& top, const Level& low, int sh,
+                                                     uint32_t (&b2)[16]) {
+  const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
+  uint32_t S2 = 0;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const uint32_t ct = codes2<BF16, DIVIDE>(x[i], top);
+    const uint32_t a = (ct >> sh) & shmask;
+    const uint32_t q = codes2<BF16, DIVIDE>(x[i], low);
+    S2 += max_s16x2(a, q) - min_s16x2(a, q);
+    b2[i] = ct | ((x[i] >> 8) & 0x00800080u);
+  }
+  return (S2 & 0xffffu) + (S2 >> 16);
+}
+
+// Bytes of one group (b2[4j + i]: elements 8j + 2i in byte 0 and 8j + 2i + 1 in byte 2) -> bit-planes:
+// on return r[k] = bit k of every byte, k < 7 code bits, k = 7 signs.
+__device__ __forceinline__ void planes_of_bytes(const uint32_t (&b2)[16], uint32_t (&r)[8]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t e = b2[4 + i] * 256u + b2[i];       // bytes: elements 2i, 8 + 2i, 2i + 1, 8 + 2i + 1
+    const uint32_t f = b2[12 + i] * 256u + b2[8 + i];  // the same, 16 further on
+    r[2 * i] = __byte_perm(e, f, 0x5410);              // byte c = element 8c + 2i
+    r[2 * i + 1] = __byte_perm(e, f, 0x7632);          // byte c = element 8c + 2i + 1
+  }
+  transpose8x32(r);
+}
+
 // Pass C on one group: codes at the chosen level as bytes (code | sign << 7), transposed into
 // bit-planes: on return r[k] = bit k of every byte, k < 7 code bits, k = 7 signs.
-template <bool BF16, int MODE>
+template <bool BF16, bool DIVIDE>
 __device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level& lv, uint32_t (&r)[8]) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     // b2 of chunk j: bytes of elements 8j + 2i (byte 0) and 8j + 2i + 1 (byte 2)
     uint32_t b2[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) b2[j] = codes2<BF16, MODE>(x[4 * j + i], lv) | ((x[4 * j + i] >> 8) & 0x00800080u);
+    for (int j = 0; j < 4; ++j) b2[j] = codes2<BF16, DIVIDE>(x[4 * j + i], lv) | ((x[4 * j + i] >> 8) & 0x00800080u);
     const uint32_t e = b2[1] * 256u + b2[0];  // bytes: elements 2i, 8 + 2i, 2i + 1, 8 + 2i + 1
     const uint32_t f = b2[3] * 256u + b2[2];  // the same, 16 further on
     r[2 * i] = __byte_perm(e, f, 0x5410);      // byte c = element 8c + 2i
     r[2 * i + 1] = __byte_perm(e, f, 0x7632);  // byte c = element 8c + 2i + 1
   }
   transpose8x32(r);
+}
+
+// The 64 bytes of group u of row `tile` into x[16] (chunks j >= nvalid lie past the end of the row: zeros).
+__device__ __forceinline__ void load_group(const EncodeParams& p, uint32_t tile, uint32_t u, uint32_t nvalid,
+                                           uint32_t (&x)[16]) {
+  const uint4* xrow = reinterpret_cast<const uint4*>(p.x + static_cast<size_t>(tile) * p.hidden);
+#pragma unroll
+  for (uint32_t j = 0; j < 4; ++j) {
+    const uint4 c = j < nvalid ? xrow[4u * u + j] : make_uint4(0u, 0u, 0u, 0u);
+    x[4 * j + 0] = c.x;
+    x[4 * j + 1] = c.y;
+    x[4 * j + 2] = c.z;
+    x[4 * j + 3] = c.w;
+  }
+}
+
+// The b* plane words of one group, in blob order (plane 0 = sign, plane 1 + k = code bit k), to dst.
+__device__ __forceinline__ void store_planes(uint32_t* dst, const uint32_t (&r)[8], int bstar, bool vec) {
+  if (vec && bstar == 8) {
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[7], r[0], r[1], r[2]);
+    reinterpret_cast<uint4*>(dst)[1] = make_uint4(r[3], r[4], r[5], r[6]);
+  } else if (vec && bstar == 4) {
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[7], r[0], r[1], r[2]);
+  } else {
+    dst[0] = r[7];
+#pragma unroll
+    for (int q = 0; q < 7; ++q) {
+      if (q < bstar - 1) dst[1 + q] = r[q];
+    }
+  }
+}
+
+// The row's min / max patterns, outlier total and per-warp outlier offsets from the per-warp partial
+// results, and the AIQ parameters of every candidate: run by one full warp, lane i takes candidate i.
+// Returns (in every lane) 1 when some level needs the division instruction.
+struct RowPartials {
+  uint32_t warp_min[32], warp_max[32], warp_cnt[32];  // warp_cnt becomes an exclusive scan
+};
+template <bool BF16>
+__device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartials& part, uint32_t nwarps, uint32_t lane,
+                                               Level* lv_out, int* S_out, uint32_t* row_cnt) {
+  using E = Elem<BF16>;
+  const uint32_t pmin = __reduce_min_sync(kFull, lane < nwarps ? part.warp_min[lane] : 0xffffu);
+  const uint32_t pmax = __reduce_max_sync(kFull, lane < nwarps ? part.warp_max[lane] : 0u);
+  const uint32_t wc = lane < nwarps ? part.warp_cnt[lane] : 0u;
+  uint32_t incl = wc;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t n = __shfl_up_sync(kFull, incl, d);
+    if (lane >= static_cast<uint32_t>(d)) incl += n;
+  }
+  part.warp_cnt[lane] = incl - wc;
+  const uint32_t total = __shfl_sync(kFull, incl, 31);
+  const Level lv = make_level(E::pattern_f32(pmin), E::pattern_f32(pmax), p.bits[min(lane, static_cast<uint32_t>(p.n_bits - 1))]);
+  if (lane < static_cast<uint32_t>(p.n_bits)) {
+    lv_out[lane] = lv;
+    S_out[lane] = 0;
+  }
+  if (lane == 0) *row_cnt = total;
+  return __all_sync(kFull, lv.packed != 0) ? 0u : 1u;
 }
 
 __device__ __forceinline__ unsigned long long pack_desc(uint32_t tag, uint32_t value) {
@@ -311,8 +344,17 @@ __device__ int resolve_prefix(const EncodeParams& p, uint32_t gen4, uint32_t til
       if (!done) {
         pos -= consumed;
         if (consumed == 0) {
-          if (++polls > kLookbackPollLimit) return TSQ_ERR_TIMEOUT;
-          __nanosleep(polls < 16u ? 100u : 500u);
+          // tile `pos` has published nothing yet: watch its two descriptors alone until it has
+          for (;;) {
+            uint32_t state = 0u;
+            if (lane == 0) {
+              state = tile_state(gen4, ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(pos)),
+                                 ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(pos) + 1));
+            }
+            if (__shfl_sync(kFull, state, 0) != 0u) break;
+            if (++polls > kLookbackPollLimit) return TSQ_ERR_TIMEOUT;
+            __nanosleep(polls < 32u ? 200u : 1000u);
+          }
         }
       }
     }
@@ -342,22 +384,71 @@ __device__ void write_header(const EncodeParams& p, unsigned long long total_wor
   h->outlier_capacity = static_cast<uint32_t>(p.lay.outlier_capacity);
 }
 
-// What the CTA shares about its row.
+// The CTA that finishes last publishes the totals and the status, and re-arms the workspace.
+__device__ void finish_call(const EncodeParams& p, uint32_t gen4) {
+  __threadfence();
+  const uint32_t prev = atomicAdd(&p.ws->done, 1u);
+  if (prev != gridDim.x - 1u) return;
+  __threadfence();
+  const uint32_t e = atomicExch(&p.ws->err, 0u);
+  // totals = the last tile's inclusive prefixes, if it got that far
+  unsigned long long tw = 0ull, to = 0ull;
+  if (p.tokens != 0u) {
+    const unsigned long long dw = ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(p.tokens - 1u));
+    const unsigned long long dout = ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(p.tokens - 1u) + 1);
+    if (tile_state(gen4, dw, dout) == kFlagPrefix) {
+      tw = static_cast<uint32_t>(dw);
+      to = static_cast<uint32_t>(dout);
+    }
+  }
+  write_header(p, tw, to);
+  reinterpret_cast<BlobHeader*>(p.blob)->status = e;
+  if (e != 0u) atomicCAS(&p.ws->enc_status, 0u, e);
+  uint32_t g = (gen4 >> 2);
+  if (g >= kGenWrap) {
+    // generation counter about to wrap: wipe the descriptors so that old tags cannot alias
+    const uint32_t n = p.ws->desc_capacity;
+    for (uint32_t i = 0; i < 2u * n; ++i) p.desc[i] = 0ull;
+    g = 0u;
+  }
+  p.ws->ticket = 0u;
+  p.ws->done = 0u;
+  p.ws->gen = g;
+}
+
+// The per-token fields of the blob, written by one thread.
+__device__ __forceinline__ void write_token_fields(const EncodeParams& p, uint32_t tile, int bstar, float scale, int zp,
+                                                   uint32_t word_end, uint32_t out_end) {
+  reinterpret_cast<uint8_t*>(p.blob + p.lay.off_bits)[tile] = static_cast<uint8_t>(bstar);
+  reinterpret_cast<float*>(p.blob + p.lay.off_scale)[tile] = scale;
+  reinterpret_cast<int32_t*>(p.blob + p.lay.off_zp)[tile] = zp;
+  uint32_t* o_word_off = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_word_off);
+  uint32_t* o_out_ptr = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_out_ptr);
+  if (tile == 0) {
+    o_word_off[0] = 0;
+    o_out_ptr[0] = 0;
+  }
+  o_word_off[tile + 1] = word_end;
+  o_out_ptr[tile + 1] = out_end;
+}
+
+// =====================================================================================================
+// encode_rows_kernel: one CTA per row, everything in order.
+// =====================================================================================================
+
 struct RowShared {
   Level lv[kMaxCand];  // lv[i]: AIQ parameters of candidate bits[i]
   int S[kMaxCand];     // distortion sum of candidate i against the top level
+  RowPartials part;
   uint32_t tile;
-  int mode;            // kFast or kDivide from the scales alone; kFast becomes kRefined when `bad` is set
-  uint32_t bad;        // some boundary of some level is not safe for the one-FMA path
-  uint32_t pmin, pmax; // patterns of the row's smallest and largest inlier magnitude
+  uint32_t divide;     // some level of the row needs the division instruction
   uint32_t row_cnt;    // outliers of the row
   uint32_t word_off, out_base;
   uint32_t status;     // TSQ_OK, or why the row is not written
-  uint32_t warp_min[32], warp_max[32], warp_cnt[32];  // per-warp partial results; warp_cnt becomes an exclusive scan
 };
 
 template <bool BF16, int UPT>
-__global__ void __launch_bounds__(1024, 1) encode_kernel(const EncodeParams p) {
+__global__ void __launch_bounds__(1024, 1) encode_rows_kernel(const EncodeParams p) {
   using E = Elem<BF16>;
   __shared__ RowShared sh;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -404,9 +495,9 @@ __global__ void __launch_bounds__(1024, 1) encode_kernel(const EncodeParams p) {
       const uint32_t mxv = __reduce_max_sync(kFull, max(mx2 & 0xffffu, mx2 >> 16));
       const uint32_t wcnt = __reduce_add_sync(kFull, cnt);
       if (lane == 0) {
-        sh.warp_min[warp] = mnv;
-        sh.warp_max[warp] = mxv;
-        sh.warp_cnt[warp] = wcnt;
+        sh.part.warp_min[warp] = mnv;
+        sh.part.warp_max[warp] = mxv;
+        sh.part.warp_cnt[warp] = wcnt;
       }
     }
     __syncthreads();
@@ -414,39 +505,11 @@ __global__ void __launch_bounds__(1024, 1) encode_kernel(const EncodeParams p) {
     // ---- AIQ parameters of every candidate level (lane i of warp 0 takes candidate i) ----
     const int bmax = p.bits[p.n_bits - 1];
     if (warp == 0) {
-      const uint32_t pmin = __reduce_min_sync(kFull, lane < nwarps ? sh.warp_min[lane] : 0xffffu);
-      const uint32_t pmax = __reduce_max_sync(kFull, lane < nwarps ? sh.warp_max[lane] : 0u);
-      // exclusive scan of the per-warp outlier counts
-      const uint32_t wc = lane < nwarps ? sh.warp_cnt[lane] : 0u;
-      uint32_t incl = wc;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t n = __shfl_up_sync(kFull, incl, d);
-        if (lane >= static_cast<uint32_t>(d)) incl += n;
-      }
-      sh.warp_cnt[lane] = incl - wc;
-      const uint32_t total = __shfl_sync(kFull, incl, 31);
-      const Level lv = make_level(E::pattern_f32(pmin), E::pattern_f32(pmax), p.bits[min(lane, static_cast<uint32_t>(p.n_bits - 1))]);
-      if (lane < static_cast<uint32_t>(p.n_bits)) {
-        sh.lv[lane] = lv;
-        sh.S[lane] = 0;
-      }
-      const bool all_fast = __all_sync(kFull, lv.fast);
-      if (lane == 0) {
-        sh.mode = all_fast ? kFast : kDivide;
-        sh.bad = 0u;
-        sh.pmin = pmin;
-        sh.pmax = pmax;
-        sh.row_cnt = total;
-      }
+      const uint32_t divide = row_levels<BF16>(p, sh.part, nwarps, lane, sh.lv, sh.S, &sh.row_cnt);
+      if (lane == 0) sh.divide = divide;
     }
     __syncthreads();
-    // ---- may the one-FMA path be trusted for this row?  every boundary of every level, all threads ----
-    if (sh.mode == kFast) {
-      if (any_boundary_disagrees<BF16>(sh.lv, p.n_bits, sh.pmin, sh.pmax, tid, blockDim.x)) sh.bad = 1u;
-      __syncthreads();
-    }
-    const int mode = (sh.mode == kFast && sh.bad != 0u) ? kRefined : sh.mode;
+    const bool divide = sh.divide != 0u;
 
     // ---- Algorithm 1: descend the candidate list while the distortion stays within tolerance ----
     const Level top = sh.lv[p.n_bits - 1];
@@ -458,9 +521,11 @@ __global__ void __launch_bounds__(1024, 1) encode_kernel(const EncodeParams p) {
       uint32_t S = 0;
 #pragma unroll
       for (int k = 0; k < UPT; ++k) {
-        S += mode == kFast      ? distortion_group<BF16, kFast>(x[k], top, low, shn)
-             : mode == kRefined ? distortion_group<BF16, kRefined>(x[k], top, low, shn)
-                                : distortion_group<BF16, kDivide>(x[k], top, low, shn);
+        if (divide) {
+          S += distortion_group<BF16, true>(x[k], top, low, shn);
+        } else {
+          S += distortion_group<BF16, false>(x[k], top, low, shn);
+        }
       }
       S = __reduce_add_sync(kFull, S);
       if (lane == 0 && S != 0u) atomicAdd(&sh.S[ci], static_cast<int>(S));
@@ -477,12 +542,10 @@ __global__ void __launch_bounds__(1024, 1) encode_kernel(const EncodeParams p) {
     uint32_t r[UPT][8];
 #pragma unroll
     for (int k = 0; k < UPT; ++k) {
-      if (mode == kFast) {
-        pack_group<BF16, kFast>(x[k], best, r[k]);
-      } else if (mode == kRefined) {
-        pack_group<BF16, kRefined>(x[k], best, r[k]);
+      if (divide) {
+        pack_group<BF16, true>(x[k], best, r[k]);
       } else {
-        pack_group<BF16, kDivide>(x[k], best, r[k]);
+        pack_group<BF16, false>(x[k], best, r[k]);
       }
     }
 
@@ -504,39 +567,14 @@ __global__ void __launch_bounds__(1024, 1) encode_kernel(const EncodeParams p) {
 
     if (sh.status == TSQ_OK) {
       const uint32_t word_off = sh.word_off, out_base = sh.out_base;
-      // ---- plane words: group u owns words u * b* .. u * b* + b* - 1, plane 0 = sign, plane 1 + k = code bit k ----
+      // ---- plane words: group u owns words u * b* .. u * b* + b* - 1 ----
       uint32_t* wrow = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_words) + word_off;
 #pragma unroll
       for (int k = 0; k < UPT; ++k) {
         const uint32_t u = UPT * tid + k;
-        if (u >= p.units) continue;
-        uint32_t* dst = wrow + static_cast<size_t>(u) * bstar;
-        if (p.vec_store && bstar == 8) {
-          reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[k][7], r[k][0], r[k][1], r[k][2]);
-          reinterpret_cast<uint4*>(dst)[1] = make_uint4(r[k][3], r[k][4], r[k][5], r[k][6]);
-        } else if (p.vec_store && bstar == 4) {
-          reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[k][7], r[k][0], r[k][1], r[k][2]);
-        } else {
-          dst[0] = r[k][7];
-#pragma unroll
-          for (int q = 0; q < 7; ++q) {
-            if (q < bstar - 1) dst[1 + q] = r[k][q];
-          }
-        }
+        if (u < p.units) store_planes(wrow + static_cast<size_t>(u) * bstar, r[k], bstar, p.vec_store != 0u);
       }
-      if (tid == 0) {
-        reinterpret_cast<uint8_t*>(p.blob + p.lay.off_bits)[tile] = static_cast<uint8_t>(bstar);
-        reinterpret_cast<float*>(p.blob + p.lay.off_scale)[tile] = best.s;
-        reinterpret_cast<int32_t*>(p.blob + p.lay.off_zp)[tile] = best.zp;
-        uint32_t* o_word_off = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_word_off);
-        uint32_t* o_out_ptr = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_out_ptr);
-        if (tile == 0) {
-          o_word_off[0] = 0;
-          o_out_ptr[0] = 0;
-        }
-        o_word_off[tile + 1] = word_off + agg_w;
-        o_out_ptr[tile + 1] = out_base + row_cnt;
-      }
+      if (tid == 0) write_token_fields(p, tile, bstar, best.s, best.zp, word_off + agg_w, out_base + row_cnt);
       // ---- CSR entries of T_above: ascending columns, original patterns (read again from the input) ----
       if (__ballot_sync(kFull, cnt != 0u) != 0u) {
         uint32_t incl = cnt;
@@ -548,7 +586,7 @@ __global__ void __launch_bounds__(1024, 1) encode_kernel(const EncodeParams p) {
         if (cnt != 0u) {
           uint32_t* o_outl = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_outl);
           const uint16_t* x16 = p.x + static_cast<size_t>(tile) * p.hidden;
-          unsigned long long at = static_cast<unsigned long long>(out_base) + sh.warp_cnt[warp] + (incl - cnt);
+          unsigned long long at = static_cast<unsigned long long>(out_base) + sh.part.warp_cnt[warp] + (incl - cnt);
           bool overflow = false;
 #pragma unroll
           for (int k = 0; k < UPT; ++k) {
@@ -571,56 +609,457 @@ __global__ void __launch_bounds__(1024, 1) encode_kernel(const EncodeParams p) {
     }
   }
 
-  // ---- the CTA that finishes last publishes the status and re-arms the workspace ----
   __syncthreads();
+  if (tid == 0) finish_call(p, gen4);
+}
+
+// =====================================================================================================
+// encode_pipe_kernel: persistent CTAs, rows in several stages at once.
+// =====================================================================================================
+// Threads: `compute` threads (one per 32-element group of a row, a multiple of 32), then the levels
+// warp, then the placement warp.  Row n of a CTA (n = 0, 1, ... in the order it takes them):
+//   compute warps, iteration n - 1  asynchronous copies of the row into xpark[n % 3], 64 bytes per thread
+//   compute warps, iteration n      pass A on the thread's own 64 bytes, thresholded values written back in
+//                                   place; per-warp partial results in meta[n % kMetaRing]
+//   levels warp                     meta[..].lv = AIQ parameters of every candidate (after a_ready > n)
+//   compute warps, iteration n + 1  passes B and C from the parked copy (after lv_ready > n), planes
+//                                   into planes[n % kRing], CSR entries into csr[n % kRing]
+//   placement warp                  offsets by look-back, bulk store of the planes, token fields, CSR
+//                                   entries (after packed > n); then placed = n + 1 frees the slots.
+// Each thread copies, thresholds and re-reads only its own group, so the parked rows need no barrier.  All counters
+// only grow; every wait on them is bounded and raises `abort`.
+
+constexpr int kRing = 4;                // rows a CTA may hold between packing and placement
+constexpr int kMetaRing = kRing + 2;    // row records: one row in pass A and one being packed on top of those
+
+struct RowMeta {
+  Level lv[kMaxCand];
+  int S[kMaxCand];
+  RowPartials part;
+  uint32_t tile, row_cnt, divide;
+  uint32_t bstar, agg_w;
+  float scale;
+  int zp;
+};
+
+struct PipeShared {
+  RowMeta meta[kMetaRing];
+  volatile uint32_t a_ready;   // rows whose pass A results are in their record
+  volatile uint32_t lv_ready;  // rows whose levels are computed
+  volatile uint32_t packed;    // rows packed and parked
+  volatile uint32_t placed;    // rows placed
+  volatile uint32_t finished;  // the compute warps are done: a_ready and packed are final
+  volatile uint32_t abort;     // a wait inside the CTA ran out
+  uint32_t next_tile[2];       // ticket of the row after the current one, by iteration parity
+};
+
+__device__ __forceinline__ void compute_barrier(uint32_t nthreads) {
+  asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
+
+// Wait until *counter > n.  Returns false when the wait is to be given up: `finished` is set and the
+// counter will not grow any more, or the CTA aborted, or the limit ran out (which raises abort).
+__device__ __forceinline__ bool wait_beyond(volatile uint32_t* counter, uint32_t n, PipeShared& sh, bool may_finish) {
+  for (uint32_t polls = 0;; ++polls) {
+    if (*counter > n) return true;
+    if (sh.abort != 0u) return false;
+    if (may_finish && sh.finished != 0u) return *counter > n;
+    if (polls > kHandshakePollLimit) {
+      sh.abort = 1u;
+      return false;
+    }
+    __nanosleep(polls < 8u ? 100u : 500u);
+  }
+}
+
+// Shared-memory address of chunk j of group u inside a parked row: the four chunks of a group are
+// rotated so that the 16-byte accesses of neighbouring threads fall into different banks.
+__device__ __forceinline__ uint32_t park_index(uint32_t u, uint32_t j) { return 4u * u + ((j + (u >> 1)) & 3u); }
+
+template <bool BF16, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodeParams p) {
+  using E = Elem<BF16>;
+  extern __shared__ __align__(128) unsigned char smem_dyn[];
+  __shared__ PipeShared sh;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const uint32_t nt = p.compute_threads, nwarps = nt >> 5;
+  const uint32_t gen4 = (*reinterpret_cast<volatile const uint32_t*>(&p.ws->gen) + 1u) << 2;
+  uint4* const xpark = reinterpret_cast<uint4*>(smem_dyn);
+  uint32_t* const planes = reinterpret_cast<uint32_t*>(smem_dyn + 3u * p.park_stride);
+  uint32_t* const csr = reinterpret_cast<uint32_t*>(smem_dyn + 3u * p.park_stride + kRing * p.planes_stride);
+
   if (tid == 0) {
-    __threadfence();
-    const uint32_t prev = atomicAdd(&p.ws->done, 1u);
-    if (prev == gridDim.x - 1u) {
-      __threadfence();
-      const uint32_t e = atomicExch(&p.ws->err, 0u);
-      // totals = the last tile's inclusive prefixes, if it got that far
-      unsigned long long tw = 0ull, to = 0ull;
-      if (p.tokens != 0u) {
-        const unsigned long long dw = ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(p.tokens - 1u));
-        const unsigned long long dout = ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(p.tokens - 1u) + 1);
-        if (tile_state(gen4, dw, dout) == kFlagPrefix) {
-          tw = static_cast<uint32_t>(dw);
-          to = static_cast<uint32_t>(dout);
+    sh.a_ready = 0u;
+    sh.lv_ready = 0u;
+    sh.packed = 0u;
+    sh.placed = 0u;
+    sh.finished = 0u;
+    sh.abort = 0u;
+    sh.next_tile[0] = atomicAdd(&p.ws->ticket, 1u);
+  }
+  __syncthreads();
+
+  if (tid < nt) {
+    // ================================ compute warps ================================
+    const uint32_t u = tid;  // this thread's group in every row
+    const uint32_t nvalid = 4u * u < p.chunks ? min(p.chunks - 4u * u, 4u) : 0u;
+    const uint32_t thr2 = p.thr16 * 0x10001u;
+    const int bmax = p.bits[p.n_bits - 1];
+    // copy of group u of row `tile` into parked row `slot`, asynchronously
+    auto fetch_row = [&](uint32_t tile, uint32_t slot) {
+      const uint4* xrow = reinterpret_cast<const uint4*>(p.x + static_cast<size_t>(tile) * p.hidden);
+      uint4* xp = xpark + slot * (p.park_stride / 16u);
+#pragma unroll
+      for (uint32_t j = 0; j < 4; ++j) {
+        if (j < nvalid) cp_async16(&xp[park_index(u, j)], &xrow[4u * u + j]);
+      }
+      cp_async_commit();
+    };
+    uint32_t tile_cur = sh.next_tile[0], tile_prev = 0u;
+    uint32_t iter = 0u;
+    bool have_prev = false;
+    uint32_t n_a = 0u;       // rows of this CTA that finished pass A
+    uint32_t n_packed = 0u;  // rows of this CTA that are packed
+    uint32_t bitmap_prev = 0u, cnt_prev = 0u;
+    if (tile_cur < p.tokens) fetch_row(tile_cur, 0u);
+
+    for (;;) {
+      const bool have_cur = tile_cur < p.tokens;
+      if (!have_cur && !have_prev) break;
+      uint32_t bitmap_cur = 0u, cnt_cur = 0u;
+      if (have_cur) {
+        // ---- pass A of row n_a: threshold split in registers, park the row, per-warp partial results ----
+        RowMeta& m = sh.meta[n_a % kMetaRing];
+        uint32_t mn2 = E::kInfPattern * 0x10001u, mx2 = 0u;
+        uint4* xp = xpark + (n_a % 3u) * (p.park_stride / 16u);
+        cp_async_wait_all();  // this thread's own copies: nobody else touches these 64 bytes
+        uint32_t x[16];
+#pragma unroll
+        for (uint32_t j = 0; j < 4; ++j) {
+          const uint4 c = j < nvalid ? xp[park_index(u, j)] : make_uint4(0u, 0u, 0u, 0u);
+          x[4 * j + 0] = c.x;
+          x[4 * j + 1] = c.y;
+          x[4 * j + 2] = c.z;
+          x[4 * j + 3] = c.w;
+        }
+        bitmap_cur = split_group<BF16>(x, nvalid, thr2, mn2, mx2);
+        cnt_cur = __popc(bitmap_cur);
+        if (bitmap_cur != 0u || nvalid < 4u) {  // outlier slots became +0 (and the chunks past the end of the row)
+#pragma unroll
+          for (uint32_t j = 0; j < 4; ++j) xp[park_index(u, j)] = make_uint4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+        }
+        const uint32_t mnv = __reduce_min_sync(kFull, min(mn2 & 0xffffu, mn2 >> 16));
+        const uint32_t mxv = __reduce_max_sync(kFull, max(mx2 & 0xffffu, mx2 >> 16));
+        const uint32_t wcnt = __reduce_add_sync(kFull, cnt_cur);
+        if (lane == 0) {
+          m.part.warp_min[warp] = mnv;
+          m.part.warp_max[warp] = mxv;
+          m.part.warp_cnt[warp] = wcnt;
         }
       }
-      write_header(p, tw, to);
-      reinterpret_cast<BlobHeader*>(p.blob)->status = e;
-      if (e != 0u) atomicCAS(&p.ws->enc_status, 0u, e);
-      uint32_t g = (gen4 >> 2);
-      if (g >= kGenWrap) {
-        // generation counter about to wrap: wipe the descriptors so that old tags cannot alias
-        const uint32_t n = p.ws->desc_capacity;
-        for (uint32_t i = 0; i < 2u * n; ++i) p.desc[i] = 0ull;
-        g = 0u;
+      if (tid == 0) {
+        if (have_cur) {
+          sh.meta[n_a % kMetaRing].tile = tile_cur;
+          sh.next_tile[(iter + 1u) & 1u] = atomicAdd(&p.ws->ticket, 1u);
+        }
+        if (have_prev) {
+          // passes B and C of row n_a - 1 need its levels, and the slot that its planes go to
+          // must have been emptied by the placement of row n_a - 1 - kRing
+          wait_beyond(&sh.lv_ready, n_a - 1u, sh, false);
+          if (n_a - 1u >= static_cast<uint32_t>(kRing)) wait_beyond(&sh.placed, n_a - 1u - kRing, sh, false);
+        }
       }
-      p.ws->ticket = 0u;
-      p.ws->done = 0u;
-      p.ws->gen = g;
+      compute_barrier(nt);
+      if (sh.abort != 0u) break;
+      if (tid == 0) {
+        __threadfence_block();
+        if (have_cur) sh.a_ready = n_a + 1u;
+        sh.packed = n_packed;
+      }
+      const uint32_t tile_next = have_cur ? sh.next_tile[(iter + 1u) & 1u] : 0xffffffffu;
+      if (tile_next < p.tokens) fetch_row(tile_next, (n_a + 1u) % 3u);  // in flight during passes B and C below
+
+      if (have_prev) {
+        const uint32_t n = n_a - 1u;
+        RowMeta& m = sh.meta[n % kMetaRing];
+        const bool divide = m.divide != 0u;
+        const uint4* xp = xpark + (n % 3u) * (p.park_stride / 16u);
+        uint32_t r[8];
+        Level best = m.lv[p.n_bits - 1];
+        int bstar = bmax;
+        {
+          uint32_t y[16];
+#pragma unroll
+          for (uint32_t j = 0; j < 4; ++j) {
+            const uint4 c = xp[park_index(u, j)];
+            y[4 * j + 0] = c.x;
+            y[4 * j + 1] = c.y;
+            y[4 * j + 2] = c.z;
+            y[4 * j + 3] = c.w;
+          }
+          if (p.n_bits == 1) {
+            if (divide) {
+              pack_group<BF16, true>(y, best, r);
+            } else {
+              pack_group<BF16, false>(y, best, r);
+            }
+          }
+        }
+        if (p.n_bits > 1) {
+          // ---- Algorithm 1: the first lower candidate, keeping the top-level bytes for pass C ----
+          const Level top = best;
+          uint32_t b2[16];
+          int ci = p.n_bits - 2;
+          {
+            uint32_t y[16];
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j) {
+              const uint4 c = xp[park_index(u, j)];
+              y[4 * j + 0] = c.x;
+              y[4 * j + 1] = c.y;
+              y[4 * j + 2] = c.z;
+              y[4 * j + 3] = c.w;
+            }
+            const Level low = m.lv[ci];
+            const int shn = bmax - p.bits[ci];
+            uint32_t S = divide ? distortion_first<BF16, true>(y, top, low, shn, b2) : distortion_first<BF16, false>(y, top, low, shn, b2);
+            S = __reduce_add_sync(kFull, S);
+            if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
+          }
+          compute_barrier(nt);
+          if (m.S[ci] > p.s_max) {
+            // delta > Delta at the first lower candidate (the usual case): the top level stays
+            planes_of_bytes(b2, r);
+          } else {
+            // ---- the descent goes on: the parked row again, one candidate at a time ----
+            uint32_t y[16];
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j) {
+              const uint4 c = xp[park_index(u, j)];
+              y[4 * j + 0] = c.x;
+              y[4 * j + 1] = c.y;
+              y[4 * j + 2] = c.z;
+              y[4 * j + 3] = c.w;
+            }
+            bstar = p.bits[ci];
+            best = m.lv[ci];
+            for (--ci; ci >= 0; --ci) {
+              const Level low = m.lv[ci];
+              const int shn = bmax - p.bits[ci];
+              uint32_t S = divide ? distortion_group<BF16, true>(y, top, low, shn) : distortion_group<BF16, false>(y, top, low, shn);
+              S = __reduce_add_sync(kFull, S);
+              if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
+              compute_barrier(nt);
+              if (m.S[ci] > p.s_max) break;  // keep the last level that passed
+              bstar = p.bits[ci];
+              best = low;
+            }
+            if (divide) {
+              pack_group<BF16, true>(y, best, r);
+            } else {
+              pack_group<BF16, false>(y, best, r);
+            }
+          }
+        }
+        const uint32_t row_cnt = m.row_cnt;
+        const uint32_t agg_w = static_cast<uint32_t>(bstar) * p.lay.wpp;
+        if (tid == 0) {
+          // the row's sizes are known: let the rows behind it see them
+          publish_aggregate(p, gen4, tile_prev, agg_w, row_cnt);
+          m.bstar = static_cast<uint32_t>(bstar);
+          m.agg_w = agg_w;
+          m.scale = best.s;
+          m.zp = best.zp;
+        }
+        // ---- planes of the chosen level into the row's slot, in blob order ----
+        if (u < p.units) store_planes(planes + (n % kRing) * (p.planes_stride / 4u) + static_cast<size_t>(u) * bstar, r, bstar, true);
+        // ---- CSR entries of T_above into the row's list: ascending columns, original patterns ----
+        if (__ballot_sync(kFull, cnt_prev != 0u) != 0u) {
+          uint32_t incl = cnt_prev;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(kFull, incl, d);
+            if (lane >= static_cast<uint32_t>(d)) incl += v;
+          }
+          if (cnt_prev != 0u && row_cnt <= p.csr_cap) {
+            uint32_t* list = csr + (n % kRing) * p.csr_cap;
+            const uint16_t* x16 = p.x + static_cast<size_t>(tile_prev) * p.hidden;
+            uint32_t at = m.part.warp_cnt[warp] + (incl - cnt_prev);
+            uint32_t bm = bitmap_prev;
+            while (bm != 0u) {
+              const uint32_t e = 32u * u + static_cast<uint32_t>(__ffs(bm) - 1);
+              bm &= bm - 1u;
+              list[at++] = (e << 16) | x16[e];
+            }
+          }
+        }
+        fence_proxy_async_smem();  // the planes are about to be read by the bulk-copy engine
+        ++n_packed;
+      }
+      have_prev = have_cur;
+      tile_prev = tile_cur;
+      bitmap_prev = bitmap_cur;
+      cnt_prev = cnt_cur;
+      if (have_cur) ++n_a;
+      tile_cur = tile_next;
+      ++iter;
     }
+    compute_barrier(nt);
+    if (tid == 0) {
+      __threadfence_block();
+      sh.packed = n_packed;
+      __threadfence_block();
+      sh.finished = 1u;
+    }
+  } else if (warp == nwarps) {
+    // ================================ levels warp ================================
+    for (uint32_t n = 0;; ++n) {
+      if (!wait_beyond(&sh.a_ready, n, sh, true)) break;
+      __threadfence_block();
+      RowMeta& m = sh.meta[n % kMetaRing];
+      const uint32_t divide = row_levels<BF16>(p, m.part, nwarps, lane, m.lv, m.S, &m.row_cnt);
+      if (lane == 0) m.divide = divide;
+      __syncwarp();
+      if (lane == 0) {
+        __threadfence_block();
+        sh.lv_ready = n + 1u;
+      }
+    }
+  } else {
+    // ================================ placement warp ================================
+    for (uint32_t n = 0;; ++n) {
+      if (!wait_beyond(&sh.packed, n, sh, true)) break;
+      __threadfence_block();
+      const RowMeta& m = sh.meta[n % kMetaRing];
+      const uint32_t tile = m.tile, agg_w = m.agg_w, row_cnt = m.row_cnt;
+      uint32_t word_off = 0, out_base = 0;
+      const int st = resolve_prefix(p, gen4, tile, agg_w, row_cnt, lane, &word_off, &out_base);
+      if (st != TSQ_OK) {
+        if (lane == 0) {
+          publish(p, gen4 | kFlagAbort, tile, 0u, 0u);
+          if (st > 0) atomicCAS(&p.ws->err, 0u, static_cast<uint32_t>(st));
+        }
+      } else {
+        uint32_t* wdst = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_words) + word_off;
+        const uint32_t* src = planes + (n % kRing) * (p.planes_stride / 4u);
+        if (p.vec_store != 0u) {
+          if (lane == 0) {
+            bulk_s2g(wdst, src, agg_w * 4u);
+            bulk_commit();
+          }
+        } else {  // runs of words that are not multiples of 16 bytes: plain stores
+          for (uint32_t w = lane; w < agg_w; w += 32) wdst[w] = src[w];
+        }
+        if (lane == 0) write_token_fields(p, tile, static_cast<int>(m.bstar), m.scale, m.zp, word_off + agg_w, out_base + row_cnt);
+        if (row_cnt != 0u) {
+          uint32_t* o_outl = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_outl);
+          bool overflow = false;
+          if (row_cnt <= p.csr_cap) {
+            const uint32_t* list = csr + (n % kRing) * p.csr_cap;
+            for (uint32_t i = lane; i < row_cnt; i += 32) {
+              const unsigned long long at = static_cast<unsigned long long>(out_base) + i;
+              if (at < p.lay.outlier_capacity) {
+                o_outl[at] = list[i];
+              } else {
+                overflow = true;
+              }
+            }
+          } else {
+            // more outliers than the list holds: take them from the input row in global memory again
+            const uint16_t* xrow = p.x + static_cast<size_t>(tile) * p.hidden;
+            unsigned long long pos = out_base;
+            for (uint32_t g = 0; g < p.units; ++g) {
+              const uint32_t e = 32u * g + lane;
+              const uint32_t raw = e < p.hidden ? xrow[e] : 0u;
+              // patterns of non-negative values order like the values; NaN patterns sort above +Inf
+              const bool out = e < p.hidden && (raw & 0x7fffu) >= p.thr16;
+              const uint32_t bal = __ballot_sync(kFull, out);
+              if (out) {
+                const unsigned long long at = pos + __popc(bal & ((1u << lane) - 1u));
+                if (at < p.lay.outlier_capacity) {
+                  o_outl[at] = (e << 16) | raw;
+                } else {
+                  overflow = true;
+                }
+              }
+              pos += __popc(bal);
+            }
+          }
+          if (__any_sync(kFull, overflow) && lane == 0) {
+            atomicCAS(&p.ws->err, 0u, static_cast<uint32_t>(TSQ_ERR_OUTLIER_OVERFLOW));
+          }
+        }
+        if (lane == 0 && p.vec_store != 0u) bulk_wait_read_all();  // the slot may be refilled after this
+      }
+      __syncwarp();
+      if (lane == 0) {
+        __threadfence_block();
+        sh.placed = n + 1u;
+      }
+    }
+    if (lane == 0) bulk_wait_all();  // shared memory must outlive the stores that read it
+  }
+
+  __syncthreads();
+  if (tid == 0) {
+    if (sh.abort != 0u) atomicCAS(&p.ws->err, 0u, static_cast<uint32_t>(TSQ_ERR_TIMEOUT));
+    finish_call(p, gen4);
   }
 }
 
 }  // namespace
 
-cudaError_t launch_encode(const EncodeParams& p, int grid, int threads, int upt, cudaStream_t stream) {
+// Two builds of the pipelined kernel: CTAs of up to 320 threads (rows of up to 8192 elements) may use
+// up to 102 registers per thread, larger CTAs up to 64.
+constexpr int kPipeSmallThreads = 320;
+
+static const void* pipe_kernel(bool bf16, int threads) {
+  if (threads <= kPipeSmallThreads) {
+    return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, kPipeSmallThreads, 2>)
+                : reinterpret_cast<const void*>(&encode_pipe_kernel<false, kPipeSmallThreads, 2>);
+  }
+  return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, 1024, 1>)
+              : reinterpret_cast<const void*>(&encode_pipe_kernel<false, 1024, 1>);
+}
+
+cudaError_t encode_pipe_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm) {
+  const void* fn = pipe_kernel(bf16, threads);
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads, smem);
+}
+
+cudaError_t launch_encode_pipe(const EncodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream) {
   const bool bf16 = p.dtype == TSQ_BF16;
-  if (upt == 1) {
+  if (threads <= kPipeSmallThreads) {
     if (bf16) {
-      encode_kernel<true, 1><<<grid, threads, 0, stream>>>(p);
+      encode_pipe_kernel<true, kPipeSmallThreads, 2><<<grid, threads, smem, stream>>>(p);
     } else {
-      encode_kernel<false, 1><<<grid, threads, 0, stream>>>(p);
+      encode_pipe_kernel<false, kPipeSmallThreads, 2><<<grid, threads, smem, stream>>>(p);
     }
   } else {
     if (bf16) {
-      encode_kernel<true, 2><<<grid, threads, 0, stream>>>(p);
+      encode_pipe_kernel<true, 1024, 1><<<grid, threads, smem, stream>>>(p);
     } else {
-      encode_kernel<false, 2><<<grid, threads, 0, stream>>>(p);
+      encode_pipe_kernel<false, 1024, 1><<<grid, threads, smem, stream>>>(p);
+    }
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_encode_rows(const EncodeParams& p, int grid, int threads, int upt, cudaStream_t stream) {
+  const bool bf16 = p.dtype == TSQ_BF16;
+  if (upt == 1) {
+    if (bf16) {
+      encode_rows_kernel<true, 1><<<grid, threads, 0, stream>>>(p);
+    } else {
+      encode_rows_kernel<false, 1><<<grid, threads, 0, stream>>>(p);
+    }
+  } else {
+    if (bf16) {
+      encode_rows_kernel<true, 2><<<grid, threads, 0, stream>>>(p);
+    } else {
+      encode_rows_kernel<false, 2><<<grid, threads, 0, stream>>>(p);
     }
   }
   return cudaGetLastError();

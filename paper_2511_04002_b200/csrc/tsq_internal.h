@@ -83,6 +83,8 @@ struct EncodeParams {
   int32_t bits[8];
   int32_t s_max;                             // floor(delta * H), clamped to [-1, INT32_MAX]
   uint32_t vec_store;                        // 1: every token's plane words start on a 16-byte boundary
+  // pipelined kernel only: thread split and shared-memory strides (bytes; csr_cap in entries)
+  uint32_t compute_threads, park_stride, planes_stride, csr_cap;
   uint32_t dtype;
   float tau, delta;
 };
@@ -97,7 +99,9 @@ struct DecodeParams {
   unsigned long long blob_bytes;
 };
 
-cudaError_t launch_encode(const EncodeParams& p, int grid, int threads, int groups_per_thread, cudaStream_t stream);
+cudaError_t launch_encode_rows(const EncodeParams& p, int grid, int threads, int groups_per_thread, cudaStream_t stream);
+cudaError_t launch_encode_pipe(const EncodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
+cudaError_t encode_pipe_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm);
 cudaError_t launch_decode(const DecodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
 cudaError_t decode_kernel_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm);
 size_t decode_smem_bytes(uint32_t row_bytes);
