@@ -20,12 +20,15 @@ __device__ __forceinline__ void record_decode_error(const DecodeParams& p, uint3
 }
 
 
-// Unpack, dequantise and stage this thread's units of one row.
-//   DIRECT = false: float(code + zp) is formed without a conversion instruction: 2^23 + n carries
-//   n in its low mantissa bits, and (2^23 + n) * s - 2^23 * s equals n * s exactly, so one FMA
-//   rounds n * s once (2^23 * s is a power-of-two multiple of s, hence exact while finite).
-//   DIRECT = true: int -> float conversion and one multiplication.
-template <bool BF16, bool DIRECT>
+// Unpack, dequantise and stage this thread's groups of one row.
+//   DIRECT = false: float(code + zp) is formed without a conversion instruction: the pattern of
+//   2^23 + n carries n in its low mantissa bits, and (2^23 + n) * s - 2^23 * s equals n * s exactly,
+//   so one FMA rounds n * s once (2^23 * s is a power-of-two multiple of s, hence exact while
+//   finite).  ZP0 (zero-point 0, the usual case) ORs the code into that pattern instead of adding.
+//   DIRECT = true: int -> float conversion and one multiplication (scales too large for 2^23 * s).
+// The integer / logic pipe is the scarce one here too: two elements travel per register, and the
+// shifts that can be multiplications are written as such.
+template <bool BF16, bool DIRECT, bool ZP0>
 __device__ __forceinline__ void restore_units(const DecodeParams& p, const uint32_t* words, uint32_t b, float s,
                                               int32_t zp) {
   using E = Elem<BF16>;
@@ -33,45 +36,51 @@ __device__ __forceinline__ void restore_units(const DecodeParams& p, const uint3
   uint4* stage4 = reinterpret_cast<uint4*>(smem_dyn);
   const float neg_bias = DIRECT ? 0.0f : -__fmul_rn(kTwo23, s);
   const bool vec = (reinterpret_cast<uintptr_t>(words) & 15u) == 0;  // 16-byte loads of a group's words
-  const uint32_t int_bias = kTwo23Bits + static_cast<uint32_t>(zp);
+  const uint32_t magic = kTwo23Bits + static_cast<uint32_t>(zp);
   for (uint32_t u = threadIdx.x; u < p.units; u += blockDim.x) {
-    // group u owns words u * b .. u * b + b - 1, one per plane
+    // group u owns words u * b .. u * b + b - 1: plane 0 = sign, plane 1 + k = code bit k.
+    // r[k] = bit k of the bytes to come: code bits in r[0..6], signs in r[7].
     uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     const uint32_t* src = words + static_cast<size_t>(u) * b;
     if (vec && b == 8u) {
       const uint4 lo = __ldg(reinterpret_cast<const uint4*>(src)), hi = __ldg(reinterpret_cast<const uint4*>(src) + 1);
-      r[0] = lo.x; r[1] = lo.y; r[2] = lo.z; r[3] = lo.w;
-      r[4] = hi.x; r[5] = hi.y; r[6] = hi.z; r[7] = hi.w;
+      r[7] = lo.x; r[0] = lo.y; r[1] = lo.z; r[2] = lo.w;
+      r[3] = hi.x; r[4] = hi.y; r[5] = hi.z; r[6] = hi.w;
     } else if (vec && b == 4u) {
       const uint4 lo = __ldg(reinterpret_cast<const uint4*>(src));
-      r[0] = lo.x; r[1] = lo.y; r[2] = lo.z; r[3] = lo.w;
+      r[7] = lo.x; r[0] = lo.y; r[1] = lo.z; r[2] = lo.w;
     } else {
+      r[7] = __ldg(src);
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        if (static_cast<uint32_t>(k) < b) r[k] = __ldg(src + k);
+      for (int k = 0; k < 7; ++k) {
+        if (static_cast<uint32_t>(k) + 1u < b) r[k] = __ldg(src + 1 + k);
       }
     }
-    transpose8x32(r);  // r[i] byte c = (code << 1 | sign) of element 8c + i
+    transpose8x32(r);  // r[i] byte c = (code | sign << 7) of element 8c + i
     const uint32_t rot = (u >> 1) & 3u;
 #pragma unroll
     for (uint32_t j = 0; j < 4; ++j) {
       const uint32_t cc = (j + rot) & 3u;
       const uint32_t cidx = 4u * u + cc;
       if (cidx >= p.chunks) continue;
-      const uint32_t shift = 8u * cc;
+      const uint32_t sel = cc * 0x1111u + 0x4400u;  // byte cc of the first operand -> byte 0, of the second -> byte 2
       uint32_t out[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint32_t blo = (r[2 * i] >> shift) & 0xffu, bhi = (r[2 * i + 1] >> shift) & 0xffu;
+        const uint32_t p2 = __byte_perm(r[2 * i], r[2 * i + 1], sel);  // elements 8cc + 2i (byte 0) and 8cc + 2i + 1 (byte 2)
+        const uint32_t clo = p2 & 0x7fu, chi = __umulhi(p2, 65536u) & 0x7fu;
         float flo, fhi;
         if (DIRECT) {
-          flo = __fmul_rn(__int2float_rn(static_cast<int>(blo >> 1) + zp), s);
-          fhi = __fmul_rn(__int2float_rn(static_cast<int>(bhi >> 1) + zp), s);
+          flo = __fmul_rn(__int2float_rn(static_cast<int>(clo) + zp), s);
+          fhi = __fmul_rn(__int2float_rn(static_cast<int>(chi) + zp), s);
+        } else if (ZP0) {
+          flo = fmaf(__uint_as_float(clo | kTwo23Bits), s, neg_bias);
+          fhi = fmaf(__uint_as_float(chi | kTwo23Bits), s, neg_bias);
         } else {
-          flo = fmaf(__uint_as_float(int_bias + (blo >> 1)), s, neg_bias);
-          fhi = fmaf(__uint_as_float(int_bias + (bhi >> 1)), s, neg_bias);
+          flo = fmaf(__uint_as_float(clo + magic), s, neg_bias);
+          fhi = fmaf(__uint_as_float(chi + magic), s, neg_bias);
         }
-        out[i] = E::pack_rn(flo, fhi) | ((blo & 1u) << 15) | ((bhi & 1u) << 31);
+        out[i] = (p2 & 0x00800080u) * 256u + E::pack_rn(flo, fhi);  // sign bits 7 / 23 -> 15 / 31
       }
       stage4[cidx] = make_uint4(out[0], out[1], out[2], out[3]);
     }
@@ -121,10 +130,12 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(const DecodeParams 
 
   const uint32_t* words = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_words) + wo;
   // 2^23 * s must stay finite for the conversion-free path; huge scales take the plain one.
-  if (s <= 0x1p100f) {
-    restore_units<BF16, false>(p, words, b, s, zp);
+  if (s > 0x1p100f) {
+    restore_units<BF16, true, false>(p, words, b, s, zp);
+  } else if (zp == 0) {
+    restore_units<BF16, false, true>(p, words, b, s, zp);
   } else {
-    restore_units<BF16, true>(p, words, b, s, zp);
+    restore_units<BF16, false, false>(p, words, b, s, zp);
   }
   __syncthreads();
 

@@ -659,7 +659,8 @@ __device__ __forceinline__ void compute_barrier(uint32_t nthreads) {
 
 // Wait until *counter > n.  Returns false when the wait is to be given up: `finished` is set and the
 // counter will not grow any more, or the CTA aborted, or the limit ran out (which raises abort).
-__device__ __forceinline__ bool wait_beyond(volatile uint32_t* counter, uint32_t n, PipeShared& sh, bool may_finish) {
+__device__ __forceinline__ bool wait_beyond(volatile uint32_t* counter, uint32_t n, PipeShared& sh, bool may_finish,
+                                            uint32_t nap_ns) {
   for (uint32_t polls = 0;; ++polls) {
     if (*counter > n) return true;
     if (sh.abort != 0u) return false;
@@ -668,7 +669,7 @@ __device__ __forceinline__ bool wait_beyond(volatile uint32_t* counter, uint32_t
       sh.abort = 1u;
       return false;
     }
-    __nanosleep(polls < 8u ? 100u : 500u);
+    __nanosleep(nap_ns);
   }
 }
 
@@ -765,8 +766,8 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         if (have_prev) {
           // passes B and C of row n_a - 1 need its levels, and the slot that its planes go to
           // must have been emptied by the placement of row n_a - 1 - kRing
-          wait_beyond(&sh.lv_ready, n_a - 1u, sh, false);
-          if (n_a - 1u >= static_cast<uint32_t>(kRing)) wait_beyond(&sh.placed, n_a - 1u - kRing, sh, false);
+          wait_beyond(&sh.lv_ready, n_a - 1u, sh, false, 100u);
+          if (n_a - 1u >= static_cast<uint32_t>(kRing)) wait_beyond(&sh.placed, n_a - 1u - kRing, sh, false, 100u);
         }
       }
       compute_barrier(nt);
@@ -914,7 +915,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
   } else if (warp == nwarps) {
     // ================================ levels warp ================================
     for (uint32_t n = 0;; ++n) {
-      if (!wait_beyond(&sh.a_ready, n, sh, true)) break;
+      if (!wait_beyond(&sh.a_ready, n, sh, true, 800u)) break;
       __threadfence_block();
       RowMeta& m = sh.meta[n % kMetaRing];
       const uint32_t divide = row_levels<BF16>(p, m.part, nwarps, lane, m.lv, m.S, &m.row_cnt);
@@ -928,7 +929,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
   } else {
     // ================================ placement warp ================================
     for (uint32_t n = 0;; ++n) {
-      if (!wait_beyond(&sh.packed, n, sh, true)) break;
+      if (!wait_beyond(&sh.packed, n, sh, true, 1500u)) break;
       __threadfence_block();
       const RowMeta& m = sh.meta[n % kMetaRing];
       const uint32_t tile = m.tile, agg_w = m.agg_w, row_cnt = m.row_cnt;
