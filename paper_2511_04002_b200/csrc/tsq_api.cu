@@ -193,7 +193,7 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
     p->pipe_csr_cap = p->units < 64u ? 64u : p->units;
     p->pipe_smem = 3u * static_cast<size_t>(p->pipe_park) + 4u * static_cast<size_t>(p->pipe_planes) + 16u * static_cast<size_t>(p->pipe_csr_cap);
     p->pipe_ctas_per_sm = 0;
-    if (ok && p->pipe_threads <= 1024 && p->pipe_smem + 8192 <= static_cast<size_t>(smem_optin)) {
+    if (ok && p->pipe_threads <= kPipeMaxThreads && p->pipe_smem + 8192 <= static_cast<size_t>(smem_optin)) {
       int blocks = 0;
       ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_threads, p->pipe_smem, &blocks) == cudaSuccess;
       p->pipe_ctas_per_sm = blocks;

@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <stdint.h>
+#include <string.h>
 
 namespace tsq {
 
@@ -97,8 +98,17 @@ struct Elem;
 template <>
 struct Elem<false> {  // IEEE binary16
   static constexpr uint32_t kInfPattern = 0x7c00u;
-  static __device__ __forceinline__ __half2 as2(uint32_t v) { return *reinterpret_cast<__half2*>(&v); }
-  static __device__ __forceinline__ uint32_t bits(__half2 v) { return *reinterpret_cast<uint32_t*>(&v); }
+  // bit casts by memcpy (a pointer cast would break the aliasing rules)
+  static __device__ __forceinline__ __half2 as2(uint32_t v) {
+    __half2 h;
+    memcpy(&h, &v, sizeof h);
+    return h;
+  }
+  static __device__ __forceinline__ uint32_t bits(__half2 v) {
+    uint32_t u;
+    memcpy(&u, &v, sizeof u);
+    return u;
+  }
   // 0xffff in each half where a >= b or the pair is unordered
   static __device__ __forceinline__ uint32_t geu_mask(uint32_t a, uint32_t b) { return __hgeu2_mask(as2(a), as2(b)); }
   static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) { return bits(__hmax2(as2(a), as2(b))); }
@@ -117,8 +127,16 @@ struct Elem<false> {  // IEEE binary16
 template <>
 struct Elem<true> {  // bfloat16
   static constexpr uint32_t kInfPattern = 0x7f80u;
-  static __device__ __forceinline__ __nv_bfloat162 as2(uint32_t v) { return *reinterpret_cast<__nv_bfloat162*>(&v); }
-  static __device__ __forceinline__ uint32_t bits(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
+  static __device__ __forceinline__ __nv_bfloat162 as2(uint32_t v) {
+    __nv_bfloat162 h;
+    memcpy(&h, &v, sizeof h);
+    return h;
+  }
+  static __device__ __forceinline__ uint32_t bits(__nv_bfloat162 v) {
+    uint32_t u;
+    memcpy(&u, &v, sizeof u);
+    return u;
+  }
   static __device__ __forceinline__ uint32_t geu_mask(uint32_t a, uint32_t b) { return __hgeu2_mask(as2(a), as2(b)); }
   static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) { return bits(__hmax2(as2(a), as2(b))); }
   static __device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) { return bits(__hmin2(as2(a), as2(b))); }

@@ -207,18 +207,21 @@ __device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level&
   transpose8x32(r);
 }
 
-// The 64 bytes of group u of row `tile` into x[16] (chunks j >= nvalid lie past the end of the row: zeros).
-__device__ __forceinline__ void load_group(const EncodeParams& p, uint32_t tile, uint32_t u, uint32_t nvalid,
-                                           uint32_t (&x)[16]) {
+// Shared-memory index of chunk j of group u inside a parked row: the four chunks of a group are
+// rotated so that the 16-byte accesses of neighbouring threads fall into different banks.
+__device__ __forceinline__ uint32_t park_index(uint32_t u, uint32_t j) { return 4u * u + ((j + (u >> 1)) & 3u); }
+
+// Asynchronous copy of the 64 bytes of group u of row `tile` into parked row `slot` (chunks
+// j >= nvalid lie past the end of the row and are not copied).
+__device__ __forceinline__ void fetch_group(const EncodeParams& p, uint4* xpark, uint32_t tile, uint32_t slot, uint32_t u,
+                                            uint32_t nvalid) {
   const uint4* xrow = reinterpret_cast<const uint4*>(p.x + static_cast<size_t>(tile) * p.hidden);
+  uint4* xp = xpark + slot * (p.park_stride / 16u);
 #pragma unroll
   for (uint32_t j = 0; j < 4; ++j) {
-    const uint4 c = j < nvalid ? xrow[4u * u + j] : make_uint4(0u, 0u, 0u, 0u);
-    x[4 * j + 0] = c.x;
-    x[4 * j + 1] = c.y;
-    x[4 * j + 2] = c.z;
-    x[4 * j + 3] = c.w;
+    if (j < nvalid) cp_async16(&xp[park_index(u, j)], &xrow[4u * u + j]);
   }
+  cp_async_commit();
 }
 
 // The b* plane words of one group, in blob order (plane 0 = sign, plane 1 + k = code bit k), to dst.
@@ -673,10 +676,6 @@ __device__ __forceinline__ bool wait_beyond(volatile uint32_t* counter, uint32_t
   }
 }
 
-// Shared-memory address of chunk j of group u inside a parked row: the four chunks of a group are
-// rotated so that the 16-byte accesses of neighbouring threads fall into different banks.
-__device__ __forceinline__ uint32_t park_index(uint32_t u, uint32_t j) { return 4u * u + ((j + (u >> 1)) & 3u); }
-
 template <bool BF16, int MAXT, int MINB>
 __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodeParams p) {
   using E = Elem<BF16>;
@@ -706,23 +705,13 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     const uint32_t nvalid = 4u * u < p.chunks ? min(p.chunks - 4u * u, 4u) : 0u;
     const uint32_t thr2 = p.thr16 * 0x10001u;
     const int bmax = p.bits[p.n_bits - 1];
-    // copy of group u of row `tile` into parked row `slot`, asynchronously
-    auto fetch_row = [&](uint32_t tile, uint32_t slot) {
-      const uint4* xrow = reinterpret_cast<const uint4*>(p.x + static_cast<size_t>(tile) * p.hidden);
-      uint4* xp = xpark + slot * (p.park_stride / 16u);
-#pragma unroll
-      for (uint32_t j = 0; j < 4; ++j) {
-        if (j < nvalid) cp_async16(&xp[park_index(u, j)], &xrow[4u * u + j]);
-      }
-      cp_async_commit();
-    };
     uint32_t tile_cur = sh.next_tile[0], tile_prev = 0u;
     uint32_t iter = 0u;
     bool have_prev = false;
     uint32_t n_a = 0u;       // rows of this CTA that finished pass A
     uint32_t n_packed = 0u;  // rows of this CTA that are packed
     uint32_t bitmap_prev = 0u, cnt_prev = 0u;
-    if (tile_cur < p.tokens) fetch_row(tile_cur, 0u);
+    if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, nvalid);
 
     for (;;) {
       const bool have_cur = tile_cur < p.tokens;
@@ -778,7 +767,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         sh.packed = n_packed;
       }
       const uint32_t tile_next = have_cur ? sh.next_tile[(iter + 1u) & 1u] : 0xffffffffu;
-      if (tile_next < p.tokens) fetch_row(tile_next, (n_a + 1u) % 3u);  // in flight during passes B and C below
+      if (tile_next < p.tokens) fetch_group(p, xpark, tile_next, (n_a + 1u) % 3u, u, nvalid);  // in flight during passes B and C below
 
       if (have_prev) {
         const uint32_t n = n_a - 1u;
@@ -1010,40 +999,27 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
 
 }  // namespace
 
-// Two builds of the pipelined kernel: CTAs of up to 320 threads (rows of up to 8192 elements) may use
-// up to 102 registers per thread, larger CTAs up to 64.
-constexpr int kPipeSmallThreads = 320;
-
-static const void* pipe_kernel(bool bf16, int threads) {
-  if (threads <= kPipeSmallThreads) {
-    return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, kPipeSmallThreads, 2>)
-                : reinterpret_cast<const void*>(&encode_pipe_kernel<false, kPipeSmallThreads, 2>);
-  }
-  return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, 1024, 1>)
-              : reinterpret_cast<const void*>(&encode_pipe_kernel<false, 1024, 1>);
+// The pipelined kernel is built for CTAs of up to kPipeMaxThreads threads (rows of up to 8192 elements)
+// and may use up to 102 registers per thread; longer rows take encode_rows_kernel.
+static const void* pipe_kernel(bool bf16) {
+  return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, kPipeMaxThreads, 2>)
+              : reinterpret_cast<const void*>(&encode_pipe_kernel<false, kPipeMaxThreads, 2>);
 }
 
 cudaError_t encode_pipe_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm) {
-  const void* fn = pipe_kernel(bf16, threads);
+  if (threads > kPipeMaxThreads) return cudaErrorInvalidValue;
+  const void* fn = pipe_kernel(bf16);
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads, smem);
 }
 
 cudaError_t launch_encode_pipe(const EncodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream) {
-  const bool bf16 = p.dtype == TSQ_BF16;
-  if (threads <= kPipeSmallThreads) {
-    if (bf16) {
-      encode_pipe_kernel<true, kPipeSmallThreads, 2><<<grid, threads, smem, stream>>>(p);
-    } else {
-      encode_pipe_kernel<false, kPipeSmallThreads, 2><<<grid, threads, smem, stream>>>(p);
-    }
+  if (threads > kPipeMaxThreads) return cudaErrorInvalidValue;
+  if (p.dtype == TSQ_BF16) {
+    encode_pipe_kernel<true, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
   } else {
-    if (bf16) {
-      encode_pipe_kernel<true, 1024, 1><<<grid, threads, smem, stream>>>(p);
-    } else {
-      encode_pipe_kernel<false, 1024, 1><<<grid, threads, smem, stream>>>(p);
-    }
+    encode_pipe_kernel<false, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
   }
   return cudaGetLastError();
 }

@@ -14,6 +14,7 @@ constexpr uint32_t kMagic = 0x31515354u;  // 'T','S','Q','1'
 constexpr uint32_t kVersion = 1u;
 constexpr int kMaxCand = 7;
 constexpr int kMaxThreads = 256;          // decoder: threads per CTA, one 32-element unit per thread per pass
+constexpr int kPipeMaxThreads = 320;      // pipelined encoder: compute threads (<= 256 groups) + two service warps
 constexpr int kEncMaxThreads = 1024;      // encoder: one CTA per row, one or two 32-element groups per thread
 
 struct BlobHeader {

@@ -46,6 +46,16 @@ def test_every_candidate_is_exercised(dtype, delta, bits):
         assert chosen == {bits[-1]}
 
 
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("shape", [(400, 10240), (330, 16384), (600, 8200), (700, 4104), (1000, 72), (450, 8192), (2000, 1024)])
+def test_many_rows_take_the_pipelined_or_the_row_kernel(dtype, shape):
+    # more rows than twice the SM count: rows of up to 8192 elements go through the pipelined kernel,
+    # longer ones through the row-at-a-time kernel
+    x = rand16(shape, dtype, seed=shape[0] * 1000 + shape[1], scale=2.0, outlier_rate=0.02)
+    x[::7] = (x[::7].float().abs() ** 3 * 0.05).to(dtype) * torch.sign(x[::7].float()).to(dtype)   # rows that descend
+    full_parity(x, 6.0, [2, 3, 4, 8], 0.2, check_cross=False)
+
+
 @pytest.mark.parametrize("hidden", [16384, 65536])
 def test_long_rows(hidden):
     x = rand16((5, hidden), torch.bfloat16, seed=hidden, scale=1.5, outlier_rate=0.001)
