@@ -90,6 +90,13 @@ __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned l
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
+// a * b + c as an integer multiply-add instruction (the FMA pipe), whatever a plain expression would become
+__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+
 // ---- packed 16-bit element operations ------------------------------------------------------------
 
 template <bool BF16>
@@ -140,7 +147,7 @@ struct Elem<true> {  // bfloat16
   static __device__ __forceinline__ uint32_t geu_mask(uint32_t a, uint32_t b) { return __hgeu2_mask(as2(a), as2(b)); }
   static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) { return bits(__hmax2(as2(a), as2(b))); }
   static __device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) { return bits(__hmin2(as2(a), as2(b))); }
-  static __device__ __forceinline__ float lo_f32(uint32_t v) { return __uint_as_float(v << 16); }
+  static __device__ __forceinline__ float lo_f32(uint32_t v) { return __uint_as_float(mad_u32(v, 65536u, 0u)); }
   static __device__ __forceinline__ float hi_f32(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
   static __device__ __forceinline__ float pattern_f32(uint32_t p) { return __uint_as_float(p << 16); }
   static __device__ __forceinline__ uint32_t pack_rn(float lo, float hi) { return bits(__floats2bfloat162_rn(lo, hi)); }

@@ -1,8 +1,8 @@
 // tsq encode kernels: threshold splitting (Eq. "ts") + token-wise TAB-Q (Algorithm 1 on AIQ,
 // Eq. "Proposed") + bit-plane packing + CSR emission, fused into one kernel.
 //
-// One CTA encodes one token row at a time, one thread per group of 32 elements.  A thread loads its
-// group's 64 bytes straight into registers, so the input is read from HBM exactly once.  The passes:
+// One CTA encodes one token row at a time, one thread per group of 32 elements (64 bytes), and every
+// thread only ever touches its own group: the input is read from HBM exactly once.  The passes:
 //   A  threshold split: outlier bitmap, outlier slots set to +0 (what T_below holds there), and
 //      the row's min / max of the inlier magnitudes (CTA reduction);
 //   B  Algorithm 1: AIQ codes at the top level and at each lower candidate, distortion sums
@@ -13,16 +13,19 @@
 // divisions) and the placement of the row's output, which has to wait for every earlier row.
 //
 // Two kernels share the passes:
-//   encode_rows_kernel  one CTA per row, everything in order; used for few rows (lowest latency per
-//                       call) and for rows too long for the pipeline's shared memory.
+//   encode_rows_kernel  one CTA per row, the group in registers from load to store, everything in
+//                       order; used for few rows (lowest latency per call) and for rows longer
+//                       than the pipelined kernel takes.
 //   encode_pipe_kernel  persistent CTAs that keep several rows in different stages at once, so that
-//                       the vector passes never wait for the scalar work or for the placement:
-//                       the compute warps run pass A of row n (parking the thresholded row in
-//                       shared memory), then passes B and C of row n - 1 from its parked copy; a
-//                       "levels" warp turns row n's min / max into AIQ parameters meanwhile; a
-//                       "placement" warp resolves the offsets of rows packed earlier, ships their
-//                       planes with one bulk asynchronous store each and writes their CSR entries.
-//                       The next row's global loads are issued before passes B and C start.
+//                       the vector passes never wait for the scalar work or for the placement.
+//                       Each compute thread copies its group of the next row into shared memory
+//                       asynchronously (no registers held), runs pass A on row n in place there,
+//                       then passes B and C of row n - 1 from its copy; a "levels" warp turns row
+//                       n's min / max into AIQ parameters meanwhile; a "placement" warp resolves the
+//                       offsets of rows packed earlier, ships their planes with one bulk
+//                       asynchronous store each and writes their CSR entries.  When the first
+//                       lower candidate fails (the usual case) pass C reuses the top-level bytes
+//                       that pass B already formed.
 //
 // The binding resource is the integer / logic pipe, which issues at half the rate of the FMA pipe:
 // the passes work on two 16-bit elements per 32-bit register wherever they can, and shifts and
@@ -97,7 +100,7 @@ __device__ __forceinline__ uint32_t codes2(uint32_t x, const Level& c) {
   const float thi = __fadd_rn(fmaf(fmaf(-q1, c.s, hi), c.r, q1), kRoundMagic);
   // pattern of 2^23 + k = 0x4B000000 + k, so thi * 2^16 + tlo (mod 2^32) = (0x4B00 + k_hi) << 16 | k_lo;
   // the constant in the high half is taken off together with zp.
-  const uint32_t k2 = __float_as_uint(thi) * 65536u + __float_as_uint(tlo);
+  const uint32_t k2 = mad_u32(__float_as_uint(thi), 65536u, __float_as_uint(tlo));
   return __viaddmin_s16x2_relu(k2, c.nz2, c.qm2);  // clamp(k - zp, 0, qmax) in both halves
 }
 
@@ -181,8 +184,8 @@ __device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], co
 __device__ __forceinline__ void planes_of_bytes(const uint32_t (&b2)[16], uint32_t (&r)[8]) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const uint32_t e = b2[4 + i] * 256u + b2[i];       // bytes: elements 2i, 8 + 2i, 2i + 1, 8 + 2i + 1
-    const uint32_t f = b2[12 + i] * 256u + b2[8 + i];  // the same, 16 further on
+    const uint32_t e = mad_u32(b2[4 + i], 256u, b2[i]);       // bytes: elements 2i, 8 + 2i, 2i + 1, 8 + 2i + 1
+    const uint32_t f = mad_u32(b2[12 + i], 256u, b2[8 + i]);  // the same, 16 further on
     r[2 * i] = __byte_perm(e, f, 0x5410);              // byte c = element 8c + 2i
     r[2 * i + 1] = __byte_perm(e, f, 0x7632);          // byte c = element 8c + 2i + 1
   }
@@ -717,6 +720,9 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       const bool have_cur = tile_cur < p.tokens;
       if (!have_cur && !have_prev) break;
       uint32_t bitmap_cur = 0u, cnt_cur = 0u;
+      // the ticket of the row after this one: asked for now, needed only after pass A
+      uint32_t ticket_next = 0xffffffffu;
+      if (tid == 0 && have_cur) ticket_next = atomicAdd(&p.ws->ticket, 1u);
       if (have_cur) {
         // ---- pass A of row n_a: threshold split in registers, park the row, per-warp partial results ----
         RowMeta& m = sh.meta[n_a % kMetaRing];
@@ -750,7 +756,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       if (tid == 0) {
         if (have_cur) {
           sh.meta[n_a % kMetaRing].tile = tile_cur;
-          sh.next_tile[(iter + 1u) & 1u] = atomicAdd(&p.ws->ticket, 1u);
+          sh.next_tile[(iter + 1u) & 1u] = ticket_next;
         }
         if (have_prev) {
           // passes B and C of row n_a - 1 need its levels, and the slot that its planes go to
@@ -904,7 +910,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
   } else if (warp == nwarps) {
     // ================================ levels warp ================================
     for (uint32_t n = 0;; ++n) {
-      if (!wait_beyond(&sh.a_ready, n, sh, true, 800u)) break;
+      if (!wait_beyond(&sh.a_ready, n, sh, true, 300u)) break;
       __threadfence_block();
       RowMeta& m = sh.meta[n % kMetaRing];
       const uint32_t divide = row_levels<BF16>(p, m.part, nwarps, lane, m.lv, m.S, &m.row_cnt);
