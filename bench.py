@@ -44,8 +44,12 @@ FALLBACK_HBM_GBS = 6650.0
 # under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
 # (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
 NCU_TRAFFIC = {
-    # "encode": {"sha256": "...", "bytes_per_token": ..., "hidden": 8192, "dtype": "bf16"},
+    "encode": {"sha256": "07b2ef0b198a92d0d7d81b14d3e63ae55a5aefa91d2a1b0ea0a91c369a468537",
+               "bytes_per_token": (134346752 + 37706496) / 8192, "hidden": 8192, "dtype": "bf16"},
+    "decode": {"sha256": "edfce2e3322f0c472a78ac4c0a93647001995ffa57ebc9cdaabb686c642990aa",
+               "bytes_per_token": (68645376 + 77305856) / 8192, "hidden": 8192, "dtype": "bf16"},
 }
+KERNEL_NAMES = {"encode": "encode_pipe_kernel (encode_rows_kernel for few or very long rows)", "decode": "decode_kernel"}
 
 
 def workload_by_name(name: str, tokens: int | None):
@@ -393,7 +397,7 @@ def run_tsq(args, w):
             same = hashlib.sha256(f.read()).hexdigest() == rec["sha256"]
         if same and rec["hidden"] == H and rec["dtype"] == w.recipe.dtype:
             traffic = rec["bytes_per_token"] * T
-    roofline = {"bound": "hbm", "kernel": "tsq %s_kernel" % dom, "achieved": kern[dom]["GB/s"], "peak": peak,
+    roofline = {"bound": "hbm", "kernel": KERNEL_NAMES[dom], "achieved": kern[dom]["GB/s"], "peak": peak,
                 "unit": "GB/s", "frac": kern[dom]["GB/s"] / peak, "traffic": traffic, "peak_source": peak_kind,
                 "bytes_per_launch": kern[dom]["bytes"], "ms_per_launch": kern[dom]["ms"],
                 "frac_of_nominal_8TBs": kern[dom]["GB/s"] / 8000.0}
