@@ -15,8 +15,7 @@
 
 #include "../tsq_encode.cu"
 
-using namespace tsq;
-
+namespace tsq {
 namespace {
 constexpr int kIters = 64;
 
@@ -77,6 +76,9 @@ __global__ void k_pass_b_c(const uint4* in, uint32_t* out, float mmax) {
   out[blockIdx.x * blockDim.x + threadIdx.x] = acc;
 }
 }  // namespace
+}  // namespace tsq
+
+using namespace tsq;
 
 int main() {
   const int blocks = 148 * 4, threads = 256, n = blocks * threads;
