@@ -190,7 +190,7 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
     p->pipe_threads = static_cast<int>(p->pipe_compute) + 64;
     p->pipe_park = p->pipe_compute * 64u;
     p->pipe_planes = (static_cast<uint32_t>(p->bmax) * p->units * 4u + 127u) & ~127u;
-    p->pipe_csr_cap = p->units < 64u ? 64u : p->units;
+    p->pipe_csr_cap = p->units < 16u ? 64u : 4u * p->units;  // one outlier in eight elements; rows above that take a slower path
     p->pipe_smem = 3u * static_cast<size_t>(p->pipe_park) + 4u * static_cast<size_t>(p->pipe_planes) + 16u * static_cast<size_t>(p->pipe_csr_cap);
     p->pipe_ctas_per_sm = 0;
     if (ok && p->pipe_threads <= kPipeMaxThreads && p->pipe_smem + 8192 <= static_cast<size_t>(smem_optin)) {

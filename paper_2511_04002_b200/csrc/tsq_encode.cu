@@ -961,24 +961,33 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
               }
             }
           } else {
-            // more outliers than the list holds: take them from the input row in global memory again
+            // more outliers than the list holds: take them from the input row in global memory again,
+            // eight groups per round trip
             const uint16_t* xrow = p.x + static_cast<size_t>(tile) * p.hidden;
             unsigned long long pos = out_base;
-            for (uint32_t g = 0; g < p.units; ++g) {
-              const uint32_t e = 32u * g + lane;
-              const uint32_t raw = e < p.hidden ? xrow[e] : 0u;
-              // patterns of non-negative values order like the values; NaN patterns sort above +Inf
-              const bool out = e < p.hidden && (raw & 0x7fffu) >= p.thr16;
-              const uint32_t bal = __ballot_sync(kFull, out);
-              if (out) {
-                const unsigned long long at = pos + __popc(bal & ((1u << lane) - 1u));
-                if (at < p.lay.outlier_capacity) {
-                  o_outl[at] = (e << 16) | raw;
-                } else {
-                  overflow = true;
-                }
+            for (uint32_t g0 = 0; g0 < p.units; g0 += 8u) {
+              uint32_t raw[8];
+#pragma unroll
+              for (uint32_t k = 0; k < 8u; ++k) {
+                const uint32_t e = 32u * (g0 + k) + lane;
+                raw[k] = e < p.hidden ? xrow[e] : 0u;
               }
-              pos += __popc(bal);
+#pragma unroll
+              for (uint32_t k = 0; k < 8u; ++k) {
+                const uint32_t e = 32u * (g0 + k) + lane;
+                // patterns of non-negative values order like the values; NaN patterns sort above +Inf
+                const bool out = e < p.hidden && (raw[k] & 0x7fffu) >= p.thr16;
+                const uint32_t bal = __ballot_sync(kFull, out);
+                if (out) {
+                  const unsigned long long at = pos + __popc(bal & ((1u << lane) - 1u));
+                  if (at < p.lay.outlier_capacity) {
+                    o_outl[at] = (e << 16) | raw[k];
+                  } else {
+                    overflow = true;
+                  }
+                }
+                pos += __popc(bal);
+              }
             }
           }
           if (__any_sync(kFull, overflow) && lane == 0) {
