@@ -962,31 +962,48 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             }
           } else {
             // more outliers than the list holds: take them from the input row in global memory again,
-            // eight groups per round trip
-            const uint16_t* xrow = p.x + static_cast<size_t>(tile) * p.hidden;
+            // 2048 elements (eight 16-byte loads per lane) per round trip
+            const uint4* xrow4 = reinterpret_cast<const uint4*>(p.x + static_cast<size_t>(tile) * p.hidden);
             unsigned long long pos = out_base;
-            for (uint32_t g0 = 0; g0 < p.units; g0 += 8u) {
-              uint32_t raw[8];
+            for (uint32_t c0 = 0; c0 < p.chunks; c0 += 256u) {
+              uint4 v[8];
 #pragma unroll
               for (uint32_t k = 0; k < 8u; ++k) {
-                const uint32_t e = 32u * (g0 + k) + lane;
-                raw[k] = e < p.hidden ? xrow[e] : 0u;
+                const uint32_t c = c0 + 32u * k + lane;
+                v[k] = c < p.chunks ? xrow4[c] : make_uint4(0u, 0u, 0u, 0u);
               }
 #pragma unroll
               for (uint32_t k = 0; k < 8u; ++k) {
-                const uint32_t e = 32u * (g0 + k) + lane;
-                // patterns of non-negative values order like the values; NaN patterns sort above +Inf
-                const bool out = e < p.hidden && (raw[k] & 0x7fffu) >= p.thr16;
-                const uint32_t bal = __ballot_sync(kFull, out);
-                if (out) {
-                  const unsigned long long at = pos + __popc(bal & ((1u << lane) - 1u));
-                  if (at < p.lay.outlier_capacity) {
-                    o_outl[at] = (e << 16) | raw[k];
-                  } else {
-                    overflow = true;
+                const uint32_t c = c0 + 32u * k + lane;  // this lane's eight elements: 8c .. 8c + 7
+                const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+                uint32_t raw[8], cnt = 0u;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  raw[j] = (j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xffffu);
+                  // patterns of non-negative values order like the values; NaN patterns sort above +Inf
+                  cnt += (c < p.chunks && (raw[j] & 0x7fffu) >= p.thr16) ? 1u : 0u;
+                }
+                uint32_t incl = cnt;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                  const uint32_t up = __shfl_up_sync(kFull, incl, d);
+                  if (lane >= static_cast<uint32_t>(d)) incl += up;
+                }
+                unsigned long long at = pos + (incl - cnt);
+                pos += __shfl_sync(kFull, incl, 31);
+                if (cnt != 0u) {
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) {
+                    if ((raw[j] & 0x7fffu) >= p.thr16) {
+                      if (at < p.lay.outlier_capacity) {
+                        o_outl[at] = ((8u * c + static_cast<uint32_t>(j)) << 16) | raw[j];
+                      } else {
+                        overflow = true;
+                      }
+                      ++at;
+                    }
                   }
                 }
-                pos += __popc(bal);
               }
             }
           }
