@@ -214,6 +214,12 @@ __device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level&
 // rotated so that the 16-byte accesses of neighbouring threads fall into different banks.
 __device__ __forceinline__ uint32_t park_index(uint32_t u, uint32_t j) { return 4u * u + ((j + (u >> 1)) & 3u); }
 
+// Number of 16-byte chunks of group u that lie inside the row (4, fewer in the last group, 0 beyond it).
+// Recomputed where it is needed: a value kept alive across the whole row loop costs a register there.
+__device__ __forceinline__ uint32_t group_chunks(const EncodeParams& p, uint32_t u) {
+  return 4u * u < p.chunks ? min(p.chunks - 4u * u, 4u) : 0u;
+}
+
 // Asynchronous copy of the 64 bytes of group u of row `tile` into parked row `slot` (chunks
 // j >= nvalid lie past the end of the row and are not copied).
 __device__ __forceinline__ void fetch_group(const EncodeParams& p, uint4* xpark, uint32_t tile, uint32_t slot, uint32_t u,
@@ -705,16 +711,11 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
   if (tid < nt) {
     // ================================ compute warps ================================
     const uint32_t u = tid;  // this thread's group in every row
-    const uint32_t nvalid = 4u * u < p.chunks ? min(p.chunks - 4u * u, 4u) : 0u;
-    const uint32_t thr2 = p.thr16 * 0x10001u;
-    const int bmax = p.bits[p.n_bits - 1];
-    uint32_t tile_cur = sh.next_tile[0], tile_prev = 0u;
-    uint32_t iter = 0u;
-    bool have_prev = false;
-    uint32_t n_a = 0u;       // rows of this CTA that finished pass A
-    uint32_t n_packed = 0u;  // rows of this CTA that are packed
+    uint32_t tile_cur = sh.next_tile[0];
+    bool have_prev = false;  // row n_a - 1 has been through pass A and is not packed yet
+    uint32_t n_a = 0u;       // rows of this CTA that finished pass A; n_a - have_prev of them are packed
     uint32_t bitmap_prev = 0u, cnt_prev = 0u;
-    if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, nvalid);
+    if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, group_chunks(p, u));
 
     for (;;) {
       const bool have_cur = tile_cur < p.tokens;
@@ -726,6 +727,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       if (have_cur) {
         // ---- pass A of row n_a: threshold split in registers, park the row, per-warp partial results ----
         RowMeta& m = sh.meta[n_a % kMetaRing];
+        const uint32_t nvalid = group_chunks(p, u);
         uint32_t mn2 = E::kInfPattern * 0x10001u, mx2 = 0u;
         uint4* xp = xpark + (n_a % 3u) * (p.park_stride / 16u);
         cp_async_wait_all();  // this thread's own copies: nobody else touches these 64 bytes
@@ -738,7 +740,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           x[4 * j + 2] = c.z;
           x[4 * j + 3] = c.w;
         }
-        bitmap_cur = split_group<BF16>(x, nvalid, thr2, mn2, mx2);
+        bitmap_cur = split_group<BF16>(x, nvalid, p.thr16 * 0x10001u, mn2, mx2);
         cnt_cur = __popc(bitmap_cur);
         if (bitmap_cur != 0u || nvalid < 4u) {  // outlier slots became +0 (and the chunks past the end of the row)
 #pragma unroll
@@ -756,7 +758,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       if (tid == 0) {
         if (have_cur) {
           sh.meta[n_a % kMetaRing].tile = tile_cur;
-          sh.next_tile[(iter + 1u) & 1u] = ticket_next;
+          sh.next_tile[(n_a + 1u) & 1u] = ticket_next;
         }
         if (have_prev) {
           // passes B and C of row n_a - 1 need its levels, and the slot that its planes go to
@@ -770,15 +772,17 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       if (tid == 0) {
         __threadfence_block();
         if (have_cur) sh.a_ready = n_a + 1u;
-        sh.packed = n_packed;
+        sh.packed = n_a - (have_prev ? 1u : 0u);
       }
-      const uint32_t tile_next = have_cur ? sh.next_tile[(iter + 1u) & 1u] : 0xffffffffu;
-      if (tile_next < p.tokens) fetch_group(p, xpark, tile_next, (n_a + 1u) % 3u, u, nvalid);  // in flight during passes B and C below
+      const uint32_t tile_next = have_cur ? sh.next_tile[(n_a + 1u) & 1u] : 0xffffffffu;
+      if (tile_next < p.tokens) fetch_group(p, xpark, tile_next, (n_a + 1u) % 3u, u, group_chunks(p, u));  // in flight during passes B and C below
 
       if (have_prev) {
         const uint32_t n = n_a - 1u;
         RowMeta& m = sh.meta[n % kMetaRing];
         const bool divide = m.divide != 0u;
+        const int bmax = p.bits[p.n_bits - 1];
+        const uint32_t tile_prev = m.tile;
         const uint4* xp = xpark + (n % 3u) * (p.park_stride / 16u);
         uint32_t r[8];
         Level best = m.lv[p.n_bits - 1];
@@ -890,20 +894,17 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           }
         }
         fence_proxy_async_smem();  // the planes are about to be read by the bulk-copy engine
-        ++n_packed;
       }
       have_prev = have_cur;
-      tile_prev = tile_cur;
       bitmap_prev = bitmap_cur;
       cnt_prev = cnt_cur;
       if (have_cur) ++n_a;
       tile_cur = tile_next;
-      ++iter;
     }
     compute_barrier(nt);
     if (tid == 0) {
       __threadfence_block();
-      sh.packed = n_packed;
+      sh.packed = n_a - (have_prev ? 1u : 0u);  // have_prev is still set only when the loop was left by an abort
       __threadfence_block();
       sh.finished = 1u;
     }
