@@ -55,7 +55,6 @@ static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 
 // In host code `g_static_ws` is only a handle for the runtime, not an address a kernel may use: the
 // device address is asked for once per device, with that device current, and kept here.
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 void* g_static_ptr[kMaxDevices] = {};
 
@@ -99,7 +98,7 @@ struct tsq_plan {
   int enc_threads, enc_upt;         // row-at-a-time encoder: CTA size and 32-element groups per thread
   // pipelined encoder: 0 CTAs per SM when the row does not fit its shared memory
   int pipe_threads, pipe_ctas_per_sm;
-  uint32_t pipe_compute, pipe_park, pipe_planes, pipe_csr_cap;
+  uint32_t pipe_compute, pipe_park, pipe_planes, pipe_csr_cap, pipe_ring;
   size_t pipe_smem;
   int sms;
   size_t dec_smem;
@@ -183,20 +182,37 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess;
   ok = ok && decode_kernel_attrs(dtype == TSQ_BF16, p->threads, p->dec_smem, &dec_blocks) == cudaSuccess;
   {
-    // pipelined encoder: three parked rows, four rows of planes and of CSR entries per CTA
+    // pipelined encoder: three parked rows and a ring of rows of planes and of CSR entries per CTA
     int smem_optin = 0;
     ok = ok && cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) == cudaSuccess;
     p->pipe_compute = (p->units + 31u) / 32u * 32u;
     p->pipe_threads = static_cast<int>(p->pipe_compute) + 64;
     p->pipe_park = p->pipe_compute * 64u;
     p->pipe_planes = (static_cast<uint32_t>(p->bmax) * p->units * 4u + 127u) & ~127u;
-    p->pipe_csr_cap = p->units < 16u ? 64u : 4u * p->units;  // one outlier in eight elements; rows above that take a slower path
-    p->pipe_smem = 3u * static_cast<size_t>(p->pipe_park) + 4u * static_cast<size_t>(p->pipe_planes) + 16u * static_cast<size_t>(p->pipe_csr_cap);
+    // a CSR list of two entries per group per ring slot (one outlier in sixteen elements; rows above that
+    // take a slower path)
+    p->pipe_csr_cap = 2u * p->pipe_compute;
+    const auto smem_for = [&](uint32_t ring) {
+      return 3u * static_cast<size_t>(p->pipe_park) + ring * (static_cast<size_t>(p->pipe_planes) + 4u * static_cast<size_t>(p->pipe_csr_cap));
+    };
+    p->pipe_ring = 4u;
+    p->pipe_smem = smem_for(p->pipe_ring);
     p->pipe_ctas_per_sm = 0;
     if (ok && p->pipe_threads <= kPipeMaxThreads && p->pipe_smem + 8192 <= static_cast<size_t>(smem_optin)) {
       int blocks = 0;
       ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_threads, p->pipe_smem, &blocks) == cudaSuccess;
       p->pipe_ctas_per_sm = blocks;
+      // the deepest ring that leaves the number of resident CTAs as it is
+      for (uint32_t ring = static_cast<uint32_t>(kMaxRing); ok && blocks > 0 && ring > 4u; --ring) {
+        if (smem_for(ring) + 8192 > static_cast<size_t>(smem_optin)) continue;
+        int b = 0;
+        ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_threads, smem_for(ring), &b) == cudaSuccess;
+        if (ok && b == blocks) {
+          p->pipe_ring = ring;
+          p->pipe_smem = smem_for(ring);
+          break;
+        }
+      }
     }
   }
   cudaSetDevice(prev_dev);
@@ -273,6 +289,7 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
     p.park_stride = plan->pipe_park;
     p.planes_stride = plan->pipe_planes;
     p.csr_cap = plan->pipe_csr_cap;
+    p.ring = plan->pipe_ring;
     const long long resident = static_cast<long long>(plan->sms) * plan->pipe_ctas_per_sm;
     const int grid = static_cast<int>(tokens < resident ? tokens : resident);
     e = launch_encode_pipe(p, grid, plan->pipe_threads, plan->pipe_smem, static_cast<cudaStream_t>(cuda_stream));

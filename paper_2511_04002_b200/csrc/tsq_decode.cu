@@ -6,6 +6,8 @@
 // Every field read from the blob is checked against the capacities of the call before it is used
 // as an index: a malformed blob makes the kernel record TSQ_ERR_CORRUPT_BLOB and skip the row.
 
+#include <mutex>
+
 #include "tsq_device.cuh"
 #include "tsq_internal.h"
 
@@ -173,8 +175,22 @@ size_t decode_smem_bytes(uint32_t row_bytes) { return (static_cast<size_t>(row_b
 cudaError_t decode_kernel_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm) {
   const void* fn = bf16 ? reinterpret_cast<const void*>(&decode_kernel<true>)
                         : reinterpret_cast<const void*>(&decode_kernel<false>);
-  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  if (e != cudaSuccess) return e;
+  // the attribute belongs to the kernel on the current device, not to a plan: it only ever grows, so
+  // that every plan can launch
+  static std::mutex mu;
+  static size_t granted[kMaxDevices][2] = {};
+  {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (smem > granted[dev][bf16 ? 1 : 0]) {
+      e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+      if (e != cudaSuccess) return e;
+      granted[dev][bf16 ? 1 : 0] = smem;
+    }
+  }
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads, smem);
 }
 

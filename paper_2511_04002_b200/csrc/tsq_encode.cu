@@ -48,6 +48,8 @@
 // whose scale is so large or so small that an intermediate product could leave the normal range,
 // or whose zero-point does not fit the packed 16-bit integer steps, use the division instruction.
 
+#include <mutex>
+
 #include "tsq_device.cuh"
 #include "tsq_internal.h"
 
@@ -252,11 +254,12 @@ __device__ __forceinline__ void store_planes(uint32_t* dst, const uint32_t (&r)[
 // The row's min / max patterns, outlier total and per-warp outlier offsets from the per-warp partial
 // results, and the AIQ parameters of every candidate: run by one full warp, lane i takes candidate i.
 // Returns (in every lane) 1 when some level needs the division instruction.
+template <int NW>  // the most warps that contribute
 struct RowPartials {
-  uint32_t warp_min[32], warp_max[32], warp_cnt[32];  // warp_cnt becomes an exclusive scan
+  uint32_t warp_min[NW], warp_max[NW], warp_cnt[NW];  // warp_cnt becomes an exclusive scan
 };
-template <bool BF16>
-__device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartials& part, uint32_t nwarps, uint32_t lane,
+template <bool BF16, int NW>
+__device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartials<NW>& part, uint32_t nwarps, uint32_t lane,
                                                Level* lv_out, int* S_out, uint32_t* row_cnt) {
   using E = Elem<BF16>;
   const uint32_t pmin = __reduce_min_sync(kFull, lane < nwarps ? part.warp_min[lane] : 0xffffu);
@@ -268,7 +271,7 @@ __device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartial
     const uint32_t n = __shfl_up_sync(kFull, incl, d);
     if (lane >= static_cast<uint32_t>(d)) incl += n;
   }
-  part.warp_cnt[lane] = incl - wc;
+  if (lane < nwarps) part.warp_cnt[lane] = incl - wc;
   const uint32_t total = __shfl_sync(kFull, incl, 31);
   const Level lv = make_level(E::pattern_f32(pmin), E::pattern_f32(pmax), p.bits[min(lane, static_cast<uint32_t>(p.n_bits - 1))]);
   if (lane < static_cast<uint32_t>(p.n_bits)) {
@@ -323,8 +326,8 @@ __device__ int resolve_prefix(const EncodeParams& p, uint32_t gen4, uint32_t til
       for (int k = 0; k < kLookbackDepth; ++k) {
         const int j = pos - (32 * k + static_cast<int>(lane));
         // before tile 0: prefix 0
-        vw[k] = j >= 0 ? ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(j)) : pack_desc(gen4 | kFlagPrefix, 0u);
-        vo[k] = j >= 0 ? ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(j) + 1) : pack_desc(gen4 | kFlagPrefix, 0u);
+        vw[k] = vo[k] = pack_desc(gen4 | kFlagPrefix, 0u);
+        if (j >= 0) ld_relaxed_u64x2(p.desc + 2 * static_cast<size_t>(j), vw[k], vo[k]);
       }
       int consumed = 32 * kLookbackDepth;
       bool stopped = false;
@@ -332,6 +335,13 @@ __device__ int resolve_prefix(const EncodeParams& p, uint32_t gen4, uint32_t til
 #pragma unroll
       for (int k = 0; k < kLookbackDepth; ++k) {
         if (stopped) continue;
+        // the usual window: 32 aggregates
+        const uint32_t agg_tag = gen4 | kFlagAggregate;
+        if (__all_sync(kFull, static_cast<uint32_t>(vw[k] >> 32) == agg_tag && static_cast<uint32_t>(vo[k] >> 32) == agg_tag)) {
+          part_w += static_cast<uint32_t>(vw[k]);
+          part_o += static_cast<uint32_t>(vo[k]);
+          continue;
+        }
         const uint32_t state = tile_state(gen4, vw[k], vo[k]);
         const uint32_t stop = __ballot_sync(kFull, state != kFlagAggregate);
         const uint32_t first = stop ? static_cast<uint32_t>(__ffs(stop) - 1) : 32u;
@@ -360,8 +370,9 @@ __device__ int resolve_prefix(const EncodeParams& p, uint32_t gen4, uint32_t til
           for (;;) {
             uint32_t state = 0u;
             if (lane == 0) {
-              state = tile_state(gen4, ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(pos)),
-                                 ld_relaxed_u64(p.desc + 2 * static_cast<size_t>(pos) + 1));
+              unsigned long long w0, w1;
+              ld_relaxed_u64x2(p.desc + 2 * static_cast<size_t>(pos), w0, w1);
+              state = tile_state(gen4, w0, w1);
             }
             if (__shfl_sync(kFull, state, 0) != 0u) break;
             if (++polls > kLookbackPollLimit) return TSQ_ERR_TIMEOUT;
@@ -451,7 +462,7 @@ __device__ __forceinline__ void write_token_fields(const EncodeParams& p, uint32
 struct RowShared {
   Level lv[kMaxCand];  // lv[i]: AIQ parameters of candidate bits[i]
   int S[kMaxCand];     // distortion sum of candidate i against the top level
-  RowPartials part;
+  RowPartials<32> part;
   uint32_t tile;
   uint32_t divide;     // some level of the row needs the division instruction
   uint32_t row_cnt;    // outliers of the row
@@ -635,19 +646,21 @@ __global__ void __launch_bounds__(1024, 1) encode_rows_kernel(const EncodeParams
 //                                   place; per-warp partial results in meta[n % kMetaRing]
 //   levels warp                     meta[..].lv = AIQ parameters of every candidate (after a_ready > n)
 //   compute warps, iteration n + 1  passes B and C from the parked copy (after lv_ready > n), planes
-//                                   into planes[n % kRing], CSR entries into csr[n % kRing]
+//                                   into planes[n % ring], CSR entries into csr[n % ring]
 //   placement warp                  offsets by look-back, bulk store of the planes, token fields, CSR
 //                                   entries (after packed > n); then placed = n + 1 frees the slots.
 // Each thread copies, thresholds and re-reads only its own group, so the parked rows need no barrier.  All counters
 // only grow; every wait on them is bounded and raises `abort`.
 
-constexpr int kRing = 4;                // rows a CTA may hold between packing and placement
-constexpr int kMetaRing = kRing + 2;    // row records: one row in pass A and one being packed on top of those
+// Rows a CTA may hold between packing and placement: p.ring (2 .. kMaxRing) slots of planes and CSR entries,
+// as many as fit beside the parked rows.  Placement waits for the rows before it, so a deep ring is what
+// keeps the compute warps busy while a slow predecessor (a row whose descent goes on) holds everybody up.
+constexpr int kMetaRing = kMaxRing + 2;  // row records: one row in pass A and one being packed on top of those
 
 struct RowMeta {
   Level lv[kMaxCand];
   int S[kMaxCand];
-  RowPartials part;
+  RowPartials<(kPipeMaxThreads - 64) / 32> part;
   uint32_t tile, row_cnt, divide;
   uint32_t bstar, agg_w;
   float scale;
@@ -695,7 +708,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
   const uint32_t gen4 = (*reinterpret_cast<volatile const uint32_t*>(&p.ws->gen) + 1u) << 2;
   uint4* const xpark = reinterpret_cast<uint4*>(smem_dyn);
   uint32_t* const planes = reinterpret_cast<uint32_t*>(smem_dyn + 3u * p.park_stride);
-  uint32_t* const csr = reinterpret_cast<uint32_t*>(smem_dyn + 3u * p.park_stride + kRing * p.planes_stride);
+  uint32_t* const csr = reinterpret_cast<uint32_t*>(smem_dyn + 3u * p.park_stride + p.ring * p.planes_stride);  // p.ring lists of p.csr_cap entries
 
   if (tid == 0) {
     sh.a_ready = 0u;
@@ -715,6 +728,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     bool have_prev = false;  // row n_a - 1 has been through pass A and is not packed yet
     uint32_t n_a = 0u;       // rows of this CTA that finished pass A; n_a - have_prev of them are packed
     uint32_t bitmap_prev = 0u, cnt_prev = 0u;
+    uint32_t slot = 0u;      // ring slot of the next row to be packed: (rows packed so far) mod p.ring
     if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, group_chunks(p, u));
 
     for (;;) {
@@ -742,7 +756,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         }
         bitmap_cur = split_group<BF16>(x, nvalid, p.thr16 * 0x10001u, mn2, mx2);
         cnt_cur = __popc(bitmap_cur);
-        if (bitmap_cur != 0u || nvalid < 4u) {  // outlier slots became +0 (and the chunks past the end of the row)
+        if (bitmap_cur != 0u || nvalid < 4u) {  // outlier slots become +0 (and the chunks past the end of the row)
 #pragma unroll
           for (uint32_t j = 0; j < 4; ++j) xp[park_index(u, j)] = make_uint4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
         }
@@ -762,9 +776,9 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         }
         if (have_prev) {
           // passes B and C of row n_a - 1 need its levels, and the slot that its planes go to
-          // must have been emptied by the placement of row n_a - 1 - kRing
+          // must have been emptied by the placement of row n_a - 1 - p.ring
           wait_beyond(&sh.lv_ready, n_a - 1u, sh, false, 100u);
-          if (n_a - 1u >= static_cast<uint32_t>(kRing)) wait_beyond(&sh.placed, n_a - 1u - kRing, sh, false, 100u);
+          if (n_a - 1u >= p.ring) wait_beyond(&sh.placed, n_a - 1u - p.ring, sh, false, 100u);
         }
       }
       compute_barrier(nt);
@@ -872,7 +886,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           m.zp = best.zp;
         }
         // ---- planes of the chosen level into the row's slot, in blob order ----
-        if (u < p.units) store_planes(planes + (n % kRing) * (p.planes_stride / 4u) + static_cast<size_t>(u) * bstar, r, bstar, true);
+        if (u < p.units) store_planes(planes + slot * (p.planes_stride / 4u) + static_cast<size_t>(u) * bstar, r, bstar, true);
         // ---- CSR entries of T_above into the row's list: ascending columns, original patterns ----
         if (__ballot_sync(kFull, cnt_prev != 0u) != 0u) {
           uint32_t incl = cnt_prev;
@@ -882,7 +896,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             if (lane >= static_cast<uint32_t>(d)) incl += v;
           }
           if (cnt_prev != 0u && row_cnt <= p.csr_cap) {
-            uint32_t* list = csr + (n % kRing) * p.csr_cap;
+            uint32_t* list = csr + slot * p.csr_cap;
             const uint16_t* x16 = p.x + static_cast<size_t>(tile_prev) * p.hidden;
             uint32_t at = m.part.warp_cnt[warp] + (incl - cnt_prev);
             uint32_t bm = bitmap_prev;
@@ -894,6 +908,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           }
         }
         fence_proxy_async_smem();  // the planes are about to be read by the bulk-copy engine
+        slot = slot + 1u == p.ring ? 0u : slot + 1u;
       }
       have_prev = have_cur;
       bitmap_prev = bitmap_cur;
@@ -924,7 +939,8 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     }
   } else {
     // ================================ placement warp ================================
-    for (uint32_t n = 0;; ++n) {
+    uint32_t slot = 0u;  // n mod p.ring
+    for (uint32_t n = 0;; ++n, slot = slot + 1u == p.ring ? 0u : slot + 1u) {
       if (!wait_beyond(&sh.packed, n, sh, true, 1500u)) break;
       __threadfence_block();
       const RowMeta& m = sh.meta[n % kMetaRing];
@@ -938,7 +954,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         }
       } else {
         uint32_t* wdst = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_words) + word_off;
-        const uint32_t* src = planes + (n % kRing) * (p.planes_stride / 4u);
+        const uint32_t* src = planes + slot * (p.planes_stride / 4u);
         if (p.vec_store != 0u) {
           if (lane == 0) {
             bulk_s2g(wdst, src, agg_w * 4u);
@@ -947,12 +963,19 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         } else {  // runs of words that are not multiples of 16 bytes: plain stores
           for (uint32_t w = lane; w < agg_w; w += 32) wdst[w] = src[w];
         }
-        if (lane == 0) write_token_fields(p, tile, static_cast<int>(m.bstar), m.scale, m.zp, word_off + agg_w, out_base + row_cnt);
+        // the token's fields, one lane each
+        if (lane == 0) reinterpret_cast<uint8_t*>(p.blob + p.lay.off_bits)[tile] = static_cast<uint8_t>(m.bstar);
+        if (lane == 1) reinterpret_cast<float*>(p.blob + p.lay.off_scale)[tile] = m.scale;
+        if (lane == 2) reinterpret_cast<int32_t*>(p.blob + p.lay.off_zp)[tile] = m.zp;
+        if (lane == 3) reinterpret_cast<uint32_t*>(p.blob + p.lay.off_word_off)[tile + 1u] = word_off + agg_w;
+        if (lane == 4) reinterpret_cast<uint32_t*>(p.blob + p.lay.off_out_ptr)[tile + 1u] = out_base + row_cnt;
+        if (tile == 0u && lane == 5) reinterpret_cast<uint32_t*>(p.blob + p.lay.off_word_off)[0] = 0u;
+        if (tile == 0u && lane == 6) reinterpret_cast<uint32_t*>(p.blob + p.lay.off_out_ptr)[0] = 0u;
         if (row_cnt != 0u) {
           uint32_t* o_outl = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_outl);
           bool overflow = false;
           if (row_cnt <= p.csr_cap) {
-            const uint32_t* list = csr + (n % kRing) * p.csr_cap;
+            const uint32_t* list = csr + slot * p.csr_cap;
             for (uint32_t i = lane; i < row_cnt; i += 32) {
               const unsigned long long at = static_cast<unsigned long long>(out_base) + i;
               if (at < p.lay.outlier_capacity) {
@@ -1012,12 +1035,15 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             atomicCAS(&p.ws->err, 0u, static_cast<uint32_t>(TSQ_ERR_OUTLIER_OVERFLOW));
           }
         }
-        if (lane == 0 && p.vec_store != 0u) bulk_wait_read_all();  // the slot may be refilled after this
       }
       __syncwarp();
       if (lane == 0) {
+        // A slot may be refilled once the bulk store has read it.  The wait is for the store of the row
+        // before this one, which has had a whole row's time to finish: this row's store is left in flight
+        // and its slot is given back one row later (plain stores have read their slot already).
+        if (p.vec_store != 0u) bulk_wait_read_but_one();
         __threadfence_block();
-        sh.placed = n + 1u;
+        sh.placed = p.vec_store != 0u ? n : n + 1u;
       }
     }
     if (lane == 0) bulk_wait_all();  // shared memory must outlive the stores that read it
@@ -1042,8 +1068,22 @@ static const void* pipe_kernel(bool bf16) {
 cudaError_t encode_pipe_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm) {
   if (threads > kPipeMaxThreads) return cudaErrorInvalidValue;
   const void* fn = pipe_kernel(bf16);
-  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  if (e != cudaSuccess) return e;
+  // the attribute belongs to the kernel on the current device, not to a plan: it only ever grows, so
+  // that every plan can launch
+  static std::mutex mu;
+  static size_t granted[kMaxDevices][2] = {};
+  {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (smem > granted[dev][bf16 ? 1 : 0]) {
+      e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+      if (e != cudaSuccess) return e;
+      granted[dev][bf16 ? 1 : 0] = smem;
+    }
+  }
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads, smem);
 }
 

@@ -15,6 +15,8 @@ constexpr uint32_t kVersion = 1u;
 constexpr int kMaxCand = 7;
 constexpr int kMaxThreads = 256;          // decoder: threads per CTA, one 32-element unit per thread per pass
 constexpr int kPipeMaxThreads = 320;      // pipelined encoder: compute threads (<= 256 groups) + two service warps
+constexpr int kMaxDevices = 64;           // devices per process that the library keeps per-device state for
+constexpr int kMaxRing = 8;               // pipelined encoder: most rows a CTA holds between packing and placement
 constexpr int kEncMaxThreads = 1024;      // encoder: one CTA per row, one or two 32-element groups per thread
 
 struct BlobHeader {
@@ -84,8 +86,8 @@ struct EncodeParams {
   int32_t bits[8];
   int32_t s_max;                             // floor(delta * H), clamped to [-1, INT32_MAX]
   uint32_t vec_store;                        // 1: every token's plane words start on a 16-byte boundary
-  // pipelined kernel only: thread split and shared-memory strides (bytes; csr_cap in entries)
-  uint32_t compute_threads, park_stride, planes_stride, csr_cap;
+  // pipelined kernel only: thread split, shared-memory strides (bytes; csr_cap in entries), ring depth in rows
+  uint32_t compute_threads, park_stride, planes_stride, csr_cap, ring;
   uint32_t dtype;
   float tau, delta;
 };
