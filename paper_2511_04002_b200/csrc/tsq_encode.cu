@@ -212,6 +212,42 @@ __device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level&
   transpose8x32(r);
 }
 
+// The same two steps for rows that need the division instruction, written as loops over the parked
+// row's words (xw: the row as 32-bit words) so that they take little room in the instruction stream.
+__device__ __forceinline__ uint32_t park_index(uint32_t u, uint32_t j);
+template <bool BF16>
+__device__ __noinline__ uint32_t rolled_distortion(const uint32_t* xw, uint32_t u, Level top, Level low, int sh) {
+  const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
+  uint32_t S = 0;
+#pragma unroll 1
+  for (uint32_t i = 0; i < 16; ++i) {
+    const uint32_t x = xw[4u * park_index(u, i >> 2) + (i & 3u)];
+    const uint32_t a = (codes2<BF16, true>(x, top) >> sh) & shmask;
+    const uint32_t q = codes2<BF16, true>(x, low);
+    const uint32_t d = max_s16x2(a, q) - min_s16x2(a, q);
+    S += (d & 0xffffu) + (d >> 16);
+  }
+  return S;
+}
+struct Planes8 {
+  uint32_t v[8];
+};
+template <bool BF16>
+__device__ __noinline__ Planes8 rolled_pack(const uint32_t* xw, uint32_t u, Level lv) {
+  uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // r[k] bit e = bit k of the byte (code | sign << 7) of element e
+#pragma unroll 1
+  for (uint32_t i = 0; i < 16; ++i) {
+    const uint32_t x = xw[4u * park_index(u, i >> 2) + (i & 3u)];
+    const uint32_t b2 = codes2<BF16, true>(x, lv) | ((x >> 8) & 0x00800080u);  // elements 2i (byte 0) and 2i + 1 (byte 2)
+#pragma unroll
+    for (int k = 0; k < 8; ++k) r[k] |= (((b2 >> k) & 1u) << (2u * i)) | (((b2 >> (16 + k)) & 1u) << (2u * i + 1u));
+  }
+  Planes8 out;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) out.v[k] = r[k];
+  return out;
+}
+
 // Shared-memory index of chunk j of group u inside a parked row: the four chunks of a group are
 // rotated so that the 16-byte accesses of neighbouring threads fall into different banks.
 __device__ __forceinline__ uint32_t park_index(uint32_t u, uint32_t j) { return 4u * u + ((j + (u >> 1)) & 3u); }
@@ -801,30 +837,29 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         uint32_t r[8];
         Level best = m.lv[p.n_bits - 1];
         int bstar = bmax;
-        {
-          uint32_t y[16];
+        const Level top = best;
+        if (divide) {
+          // ---- a row whose scale or zero-point is outside the range of the FMA quotient and of the packed
+          //      integer steps (rare): Algorithm 1 with the division instruction, in loops that are not unrolled ----
+          const uint32_t* xw = reinterpret_cast<const uint32_t*>(xp);
+          for (int ci = p.n_bits - 2; ci >= 0; --ci) {
+            const Level low = m.lv[ci];
+            uint32_t S = rolled_distortion<BF16>(xw, u, top, low, bmax - p.bits[ci]);
+            S = __reduce_add_sync(kFull, S);
+            if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
+            compute_barrier(nt);
+            if (m.S[ci] > p.s_max) break;  // keep the last level that passed
+            bstar = p.bits[ci];
+            best = low;
+          }
+          const Planes8 pl = rolled_pack<BF16>(xw, u, best);
 #pragma unroll
-          for (uint32_t j = 0; j < 4; ++j) {
-            const uint4 c = xp[park_index(u, j)];
-            y[4 * j + 0] = c.x;
-            y[4 * j + 1] = c.y;
-            y[4 * j + 2] = c.z;
-            y[4 * j + 3] = c.w;
-          }
-          if (p.n_bits == 1) {
-            if (divide) {
-              pack_group<BF16, true>(y, best, r);
-            } else {
-              pack_group<BF16, false>(y, best, r);
-            }
-          }
-        }
-        if (p.n_bits > 1) {
-          // ---- Algorithm 1: the first lower candidate, keeping the top-level bytes for pass C ----
-          const Level top = best;
+          for (int k = 0; k < 8; ++k) r[k] = pl.v[k];
+        } else {
+          // ---- Algorithm 1, one candidate per turn; every turn also forms the top-level bytes, which
+          //      pass C takes over when the first lower candidate fails (the usual case) ----
           uint32_t b2[16];
-          int ci = p.n_bits - 2;
-          {
+          for (int ci = p.n_bits - 2; ci >= 0; --ci) {
             uint32_t y[16];
 #pragma unroll
             for (uint32_t j = 0; j < 4; ++j) {
@@ -835,17 +870,18 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
               y[4 * j + 3] = c.w;
             }
             const Level low = m.lv[ci];
-            const int shn = bmax - p.bits[ci];
-            uint32_t S = divide ? distortion_first<BF16, true>(y, top, low, shn, b2) : distortion_first<BF16, false>(y, top, low, shn, b2);
+            uint32_t S = distortion_first<BF16, false>(y, top, low, bmax - p.bits[ci], b2);
             S = __reduce_add_sync(kFull, S);
             if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
+            compute_barrier(nt);
+            if (m.S[ci] > p.s_max) break;  // keep the last level that passed
+            bstar = p.bits[ci];
+            best = low;
           }
-          compute_barrier(nt);
-          if (m.S[ci] > p.s_max) {
-            // delta > Delta at the first lower candidate (the usual case): the top level stays
+          if (p.n_bits > 1 && bstar == bmax) {
             planes_of_bytes(b2, r);
           } else {
-            // ---- the descent goes on: the parked row again, one candidate at a time ----
+            // a lower level was chosen (or there is one candidate only): the parked row once more
             uint32_t y[16];
 #pragma unroll
             for (uint32_t j = 0; j < 4; ++j) {
@@ -855,24 +891,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
               y[4 * j + 2] = c.z;
               y[4 * j + 3] = c.w;
             }
-            bstar = p.bits[ci];
-            best = m.lv[ci];
-            for (--ci; ci >= 0; --ci) {
-              const Level low = m.lv[ci];
-              const int shn = bmax - p.bits[ci];
-              uint32_t S = divide ? distortion_group<BF16, true>(y, top, low, shn) : distortion_group<BF16, false>(y, top, low, shn);
-              S = __reduce_add_sync(kFull, S);
-              if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
-              compute_barrier(nt);
-              if (m.S[ci] > p.s_max) break;  // keep the last level that passed
-              bstar = p.bits[ci];
-              best = low;
-            }
-            if (divide) {
-              pack_group<BF16, true>(y, best, r);
-            } else {
-              pack_group<BF16, false>(y, best, r);
-            }
+            pack_group<BF16, false>(y, best, r);
           }
         }
         const uint32_t row_cnt = m.row_cnt;
