@@ -56,6 +56,24 @@ def test_many_rows_take_the_pipelined_or_the_row_kernel(dtype, shape):
     full_parity(x, 6.0, [2, 3, 4, 8], 0.2, check_cross=False)
 
 
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("shape", [(500, 4096), (420, 8192), (900, 264)])
+@pytest.mark.parametrize("delta", [0.2, 1e9])
+def test_many_rows_some_needing_the_division_instruction(dtype, shape, delta):
+    # the pipelined kernel's rolled path: rows whose zero-point is large (a narrow range far from zero) and,
+    # for bf16, rows whose scale is far outside the range of the FMA quotient, among ordinary rows
+    T, H = shape
+    x = rand16(shape, dtype, seed=T * 31 + H, scale=1.5, outlier_rate=0.0).float()
+    g = torch.Generator().manual_seed(T + H)
+    x[::5] = 100.0 + torch.rand((x[::5].shape[0], H), generator=g)                    # zero-point 12700: past the packed steps
+    x[4::5] = 100.0 + torch.rand((x[4::5].shape[0], H), generator=g) * 0.0625         # fp16: zero-point 203200; bf16: a constant row
+    x[1::5] = -(3.0 + torch.rand((x[1::5].shape[0], H), generator=g) * 0.25)          # zero-point of a few thousand: packed steps
+    if dtype == torch.bfloat16:
+        x[2::11] *= 1e37
+        x[3::13] *= 1e-36
+    full_parity(x.to(dtype).contiguous(), INF, [2, 3, 4, 8], delta, check_cross=False)
+
+
 @pytest.mark.parametrize("hidden", [16384, 65536])
 def test_long_rows(hidden):
     x = rand16((5, hidden), torch.bfloat16, seed=hidden, scale=1.5, outlier_rate=0.001)
