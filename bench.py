@@ -44,10 +44,10 @@ FALLBACK_HBM_GBS = 6650.0
 # under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
 # (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
 NCU_TRAFFIC = {
-    "encode": {"sha256": "07b2ef0b198a92d0d7d81b14d3e63ae55a5aefa91d2a1b0ea0a91c369a468537",
-               "bytes_per_token": (134346752 + 37706496) / 8192, "hidden": 8192, "dtype": "bf16"},
-    "decode": {"sha256": "edfce2e3322f0c472a78ac4c0a93647001995ffa57ebc9cdaabb686c642990aa",
-               "bytes_per_token": (68645376 + 77305856) / 8192, "hidden": 8192, "dtype": "bf16"},
+    "encode": {"sha256": "3450ee45b9461d6379551de2741a58b9f554c33b715037b325203cd8ad733b22",
+               "bytes_per_token": (134338560 + 37416192) / 8192, "hidden": 8192, "dtype": "bf16"},
+    "decode": {"sha256": "be5a19566be9449ea9a692b638af3c35bae99b39688b20c4117b9328b6eaedf3",
+               "bytes_per_token": (68643840 + 77444608) / 8192, "hidden": 8192, "dtype": "bf16"},
 }
 KERNEL_NAMES = {"encode": "encode_pipe_kernel (encode_rows_kernel for few or very long rows)", "decode": "decode_kernel"}
 
