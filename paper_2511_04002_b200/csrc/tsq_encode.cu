@@ -62,14 +62,15 @@ constexpr uint32_t kLookbackPollLimit = 1u << 20;
 constexpr uint32_t kHandshakePollLimit = 1u << 22;
 
 // AIQ parameters of one candidate level for one row (Eq. "Proposed").
-struct Level {
+struct __align__(16) Level {  // 32 bytes: what the usual path reads comes first, in one 16-byte load
   float s;       // scale
   float r;       // fl(1 / s)
-  int zp;        // zero-point rint(m_min / s)
-  int qmax;      // 2^(b-1) - 1
   uint32_t nz2;  // -zp in the low half, -zp - kRoundMagicHi in the high half (see codes2)
   uint32_t qm2;  // qmax in both 16-bit halves
+  int zp;        // zero-point rint(m_min / s)
+  int qmax;      // 2^(b-1) - 1
   int packed;    // scale and zero-point in the range where the FMA quotient and the packed steps are safe
+  int pad;
 };
 
 __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
@@ -82,6 +83,7 @@ __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
   c.nz2 = (static_cast<uint32_t>(-c.zp) & 0xffffu) | (static_cast<uint32_t>(-c.zp - static_cast<int>(kRoundMagicHi)) << 16);
   c.qm2 = static_cast<uint32_t>(c.qmax) * 0x10001u;
   // rint(m / s) <= zp + qmax + 1 must stay a small positive 16-bit integer for the packed steps
+  c.pad = 0;
   c.packed = ((c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && (c.zp < 12000)) ? 1 : 0;
   return c;
 }
