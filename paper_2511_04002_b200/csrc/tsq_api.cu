@@ -94,7 +94,8 @@ struct tsq_plan {
   int32_t bmax;
   int32_t s_max;
   uint32_t thr16;
-  int threads;                      // decoder CTA size
+  int threads;                      // decoder CTA size, one group per thread
+  int threads_half, dec_blocks_half; // the same with two groups per thread, and its resident CTAs per SM
   int enc_threads, enc_upt;         // row-at-a-time encoder: CTA size and 32-element groups per thread
   // pipelined encoder: 0 CTAs per SM when the row does not fit its shared memory
   int pipe_threads, pipe_ctas_per_sm;
@@ -161,8 +162,19 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   const double smax = std::floor(static_cast<double>(delta) * static_cast<double>(hidden));
   p->s_max = smax < -1.0 ? -1 : (smax > 2147483647.0 ? 2147483647 : static_cast<int32_t>(smax));
   p->thr16 = threshold_pattern(dtype, tau);
+  // decoder CTA: one 32-element group per thread, or two when the call has rows enough to fill the device
+  // several times over with the smaller CTAs (a thread's fixed work, checking the header and the token's
+  // fields, is then spread over 64 elements: 8 % faster at 8192 x 8192 and 32768 x 4096; with fewer rows
+  // the smaller CTAs leave the device short of threads and are slower); never fewer than 64 threads while
+  // the row has that many groups
   p->threads = static_cast<int>(((p->units + 31u) / 32u) * 32u);
   if (p->threads > kMaxThreads) p->threads = kMaxThreads;
+  {
+    const uint32_t all = static_cast<uint32_t>(p->threads), half = (((p->units + 1u) / 2u + 31u) / 32u) * 32u;
+    const uint32_t floor64 = all < 64u ? all : 64u;
+    p->threads_half = static_cast<int>(half > floor64 ? half : floor64);
+    if (p->threads_half > p->threads) p->threads_half = p->threads;
+  }
   // encoder: one thread per 32-element group, two for rows longer than kEncMaxThreads groups
   p->enc_upt = p->units > static_cast<uint32_t>(kEncMaxThreads) ? 2 : 1;
   p->enc_threads = static_cast<int>(((p->units + p->enc_upt - 1) / p->enc_upt + 31u) / 32u * 32u);
@@ -181,6 +193,7 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   int sms = 0, dec_blocks = 0;
   ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess;
   ok = ok && decode_kernel_attrs(dtype == TSQ_BF16, p->threads, p->dec_smem, &dec_blocks) == cudaSuccess;
+  ok = ok && decode_kernel_attrs(dtype == TSQ_BF16, p->threads_half, p->dec_smem, &p->dec_blocks_half) == cudaSuccess;
   {
     // pipelined encoder: three parked rows and a ring of rows of planes and of CSR entries per CTA
     int smem_optin = 0;
@@ -326,8 +339,9 @@ tsq_status_t tsq_decode(const tsq_plan_t* plan, const void* blob_dev, size_t blo
   p.bmax = static_cast<uint32_t>(plan->bmax);
   p.dtype = static_cast<uint32_t>(plan->dtype);
   p.blob_bytes = blob_bytes;
-  const cudaError_t e = launch_decode(p, static_cast<int>(tokens), plan->threads, plan->dec_smem,
-                                      static_cast<cudaStream_t>(cuda_stream));
+  const bool many_rows = tokens >= 3 * static_cast<int64_t>(plan->sms) * plan->dec_blocks_half;
+  const cudaError_t e = launch_decode(p, static_cast<int>(tokens), many_rows ? plan->threads_half : plan->threads,
+                                      plan->dec_smem, static_cast<cudaStream_t>(cuda_stream));
   g_launches.fetch_add(1);
   return e == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
 }
