@@ -771,14 +771,14 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     uint32_t tile_cur = sh.next_tile[0];
     bool have_prev = false;  // row n_a - 1 has been through pass A and is not packed yet
     uint32_t n_a = 0u;       // rows of this CTA that finished pass A; n_a - have_prev of them are packed
-    uint32_t bitmap_prev = 0u, cnt_prev = 0u;
+    uint32_t bitmap_prev = 0u, cnt_prev = 0u, first_prev = 0u;  // outliers of the thread's group in row n_a - 1
     uint32_t slot = 0u;      // ring slot of the next row to be packed: (rows packed so far) mod p.ring
     if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, group_chunks(p, u));
 
     for (;;) {
       const bool have_cur = tile_cur < p.tokens;
       if (!have_cur && !have_prev) break;
-      uint32_t bitmap_cur = 0u, cnt_cur = 0u;
+      uint32_t bitmap_cur = 0u, cnt_cur = 0u, first_cur = 0u;
       // the ticket of the row after this one: asked for now, needed only after pass A
       uint32_t ticket_next = 0xffffffffu;
       if (tid == 0 && have_cur) ticket_next = atomicAdd(&p.ws->ticket, 1u);
@@ -800,6 +800,12 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         }
         bitmap_cur = split_group<BF16>(x, nvalid, p.thr16 * 0x10001u, mn2, mx2);
         cnt_cur = __popc(bitmap_cur);
+        if (bitmap_cur != 0u) {
+          // the original pattern of the group's first outlier, from the parked row while it still holds it:
+          // the CSR entry is written an iteration later, and most groups with an outlier have just one
+          const uint32_t b = static_cast<uint32_t>(__ffs(bitmap_cur) - 1);
+          first_cur = reinterpret_cast<const uint16_t*>(xp)[8u * park_index(nt, u, b >> 3) + (b & 7u)];
+        }
         if (bitmap_cur != 0u || nvalid < 4u) {  // outlier slots become +0 (and the chunks past the end of the row)
 #pragma unroll
           for (uint32_t j = 0; j < 4; ++j) xp[park_index(nt, u, j)] = make_uint4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
@@ -934,7 +940,9 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             const uint16_t* x16 = p.x + static_cast<size_t>(tile_prev) * p.hidden;
             uint32_t at = m.part.warp_cnt[warp] + before;
             uint32_t bm = bitmap_prev;
-            while (bm != 0u) {
+            list[at++] = ((32u * u + static_cast<uint32_t>(__ffs(bm) - 1)) << 16) | first_prev;
+            bm &= bm - 1u;
+            while (bm != 0u) {  // further outliers of the group: read from the input again
               const uint32_t e = 32u * u + static_cast<uint32_t>(__ffs(bm) - 1);
               bm &= bm - 1u;
               list[at++] = (e << 16) | x16[e];
@@ -947,6 +955,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       have_prev = have_cur;
       bitmap_prev = bitmap_cur;
       cnt_prev = cnt_cur;
+      first_prev = first_cur;
       if (have_cur) ++n_a;
       tile_cur = tile_next;
     }
