@@ -774,14 +774,15 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     uint32_t bitmap_prev = 0u, cnt_prev = 0u, first_prev = 0u;  // outliers of the thread's group in row n_a - 1
     uint32_t slot = 0u;      // ring slot of the next row to be packed: (rows packed so far) mod p.ring
     if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, group_chunks(p, u));
+    // thread 0: the ticket of the row after tile_cur, asked for a whole iteration before it is needed
+    // (the round trip of the atomic is longer than pass A)
+    uint32_t ticket_ahead = 0xffffffffu;
+    if (tid == 0 && tile_cur < p.tokens) ticket_ahead = atomicAdd(&p.ws->ticket, 1u);
 
     for (;;) {
       const bool have_cur = tile_cur < p.tokens;
       if (!have_cur && !have_prev) break;
       uint32_t bitmap_cur = 0u, cnt_cur = 0u, first_cur = 0u;
-      // the ticket of the row after this one: asked for now, needed only after pass A
-      uint32_t ticket_next = 0xffffffffu;
-      if (tid == 0 && have_cur) ticket_next = atomicAdd(&p.ws->ticket, 1u);
       if (have_cur) {
         // ---- pass A of row n_a: threshold split in registers, park the row, per-warp partial results ----
         RowMeta& m = sh.meta[n_a % kMetaRing];
@@ -822,7 +823,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       if (tid == 0) {
         if (have_cur) {
           sh.meta[n_a % kMetaRing].tile = tile_cur;
-          sh.next_tile[(n_a + 1u) & 1u] = ticket_next;
+          sh.next_tile[(n_a + 1u) & 1u] = ticket_ahead;
         }
         if (have_prev) {
           // passes B and C of row n_a - 1 need its levels, and the slot that its planes go to
@@ -837,6 +838,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         __threadfence_block();
         if (have_cur) sh.a_ready = n_a + 1u;
         sh.packed = n_a - (have_prev ? 1u : 0u);
+        if (have_cur && ticket_ahead < p.tokens) ticket_ahead = atomicAdd(&p.ws->ticket, 1u);  // for the row after the next
       }
       const uint32_t tile_next = have_cur ? sh.next_tile[(n_a + 1u) & 1u] : 0xffffffffu;
       if (tile_next < p.tokens) fetch_group(p, xpark, tile_next, (n_a + 1u) % 3u, u, group_chunks(p, u));  // in flight during passes B and C below
