@@ -99,6 +99,7 @@ struct tsq_plan {
   int enc_threads, enc_upt;         // row-at-a-time encoder: CTA size and 32-element groups per thread
   // pipelined encoder: 0 CTAs per SM when the row does not fit its shared memory
   int pipe_threads, pipe_ctas_per_sm;
+  bool pipe_full;
   uint32_t pipe_compute, pipe_park, pipe_planes, pipe_csr_cap, pipe_ring;
   size_t pipe_smem;
   int sms;
@@ -199,6 +200,7 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
     int smem_optin = 0;
     ok = ok && cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) == cudaSuccess;
     p->pipe_compute = (p->units + 31u) / 32u * 32u;
+    p->pipe_full = (p->hidden % 32u == 0u) && (p->units == p->pipe_compute);  // every compute thread owns a whole group
     p->pipe_threads = static_cast<int>(p->pipe_compute) + 64;
     p->pipe_park = p->pipe_compute * 64u;
     p->pipe_planes = (static_cast<uint32_t>(p->bmax) * p->units * 4u + 127u) & ~127u;
@@ -213,13 +215,13 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
     p->pipe_ctas_per_sm = 0;
     if (ok && p->pipe_threads <= kPipeMaxThreads && p->pipe_smem + 8192 <= static_cast<size_t>(smem_optin)) {
       int blocks = 0;
-      ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_threads, p->pipe_smem, &blocks) == cudaSuccess;
+      ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, p->pipe_threads, p->pipe_smem, &blocks) == cudaSuccess;
       p->pipe_ctas_per_sm = blocks;
       // the deepest ring that leaves the number of resident CTAs as it is
       for (uint32_t ring = static_cast<uint32_t>(kMaxRing); ok && blocks > 0 && ring > 4u; --ring) {
         if (smem_for(ring) + 8192 > static_cast<size_t>(smem_optin)) continue;
         int b = 0;
-        ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_threads, smem_for(ring), &b) == cudaSuccess;
+        ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, p->pipe_threads, smem_for(ring), &b) == cudaSuccess;
         if (ok && b == blocks) {
           p->pipe_ring = ring;
           p->pipe_smem = smem_for(ring);
@@ -305,7 +307,7 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
     p.ring = plan->pipe_ring;
     const long long resident = static_cast<long long>(plan->sms) * plan->pipe_ctas_per_sm;
     const int grid = static_cast<int>(tokens < resident ? tokens : resident);
-    e = launch_encode_pipe(p, grid, plan->pipe_threads, plan->pipe_smem, static_cast<cudaStream_t>(cuda_stream));
+    e = launch_encode_pipe(p, plan->pipe_full, grid, plan->pipe_threads, plan->pipe_smem, static_cast<cudaStream_t>(cuda_stream));
   } else {
     // few rows (or rows too long for the pipeline): one CTA per row; a call without rows still launches
     // one CTA, which writes the header

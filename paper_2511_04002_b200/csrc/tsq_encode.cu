@@ -742,7 +742,9 @@ __device__ __forceinline__ bool wait_beyond(volatile uint32_t* counter, uint32_t
   }
 }
 
-template <bool BF16, int MAXT, int MINB>
+// FULL: every compute thread owns a whole 32-element group (hidden is a multiple of 1024), so none of the
+// checks for short or missing groups is needed.
+template <bool BF16, bool FULL, int MAXT, int MINB>
 __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodeParams p) {
   using E = Elem<BF16>;
   extern __shared__ __align__(128) unsigned char smem_dyn[];
@@ -773,7 +775,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     uint32_t n_a = 0u;       // rows of this CTA that finished pass A; n_a - have_prev of them are packed
     uint32_t bitmap_prev = 0u, cnt_prev = 0u, first_prev = 0u;  // outliers of the thread's group in row n_a - 1
     uint32_t slot = 0u;      // ring slot of the next row to be packed: (rows packed so far) mod p.ring
-    if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, group_chunks(p, u));
+    if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, FULL ? 4u : group_chunks(p, u));
     // thread 0: the ticket of the row after tile_cur, asked for a whole iteration before it is needed
     // (the round trip of the atomic is longer than pass A)
     uint32_t ticket_ahead = 0xffffffffu;
@@ -786,7 +788,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       if (have_cur) {
         // ---- pass A of row n_a: threshold split in registers, park the row, per-warp partial results ----
         RowMeta& m = sh.meta[n_a % kMetaRing];
-        const uint32_t nvalid = group_chunks(p, u);
+        const uint32_t nvalid = FULL ? 4u : group_chunks(p, u);
         uint32_t mn2 = E::kInfPattern * 0x10001u, mx2 = 0u;
         uint4* xp = xpark + (n_a % 3u) * (p.park_stride / 16u);
         cp_async_wait_all();  // this thread's own copies: nobody else touches these 64 bytes
@@ -841,7 +843,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         if (have_cur && ticket_ahead < p.tokens) ticket_ahead = atomicAdd(&p.ws->ticket, 1u);  // for the row after the next
       }
       const uint32_t tile_next = have_cur ? sh.next_tile[(n_a + 1u) & 1u] : 0xffffffffu;
-      if (tile_next < p.tokens) fetch_group(p, xpark, tile_next, (n_a + 1u) % 3u, u, group_chunks(p, u));  // in flight during passes B and C below
+      if (tile_next < p.tokens) fetch_group(p, xpark, tile_next, (n_a + 1u) % 3u, u, FULL ? 4u : group_chunks(p, u));  // in flight during passes B and C below
 
       if (have_prev) {
         const uint32_t n = n_a - 1u;
@@ -921,7 +923,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           m.zp = best.zp;
         }
         // ---- planes of the chosen level into the row's slot, in blob order ----
-        if (u < p.units) store_planes(planes + slot * (p.planes_stride / 4u) + static_cast<size_t>(u) * bstar, r, bstar, true);
+        if (FULL || u < p.units) store_planes(planes + slot * (p.planes_stride / 4u) + u * static_cast<uint32_t>(bstar), r, bstar, true);
         // ---- CSR entries of T_above into the row's list: ascending columns, original patterns ----
         const uint32_t flagged = __ballot_sync(kFull, cnt_prev != 0u);
         if (flagged != 0u) {
@@ -1105,39 +1107,50 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
 
 // The pipelined kernel is built for CTAs of up to kPipeMaxThreads threads (rows of up to 8192 elements)
 // and may use up to 102 registers per thread; longer rows take encode_rows_kernel.
-static const void* pipe_kernel(bool bf16) {
-  return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, kPipeMaxThreads, 2>)
-              : reinterpret_cast<const void*>(&encode_pipe_kernel<false, kPipeMaxThreads, 2>);
+static const void* pipe_kernel(bool bf16, bool full) {
+  if (full) {
+    return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, true, kPipeMaxThreads, 2>)
+                : reinterpret_cast<const void*>(&encode_pipe_kernel<false, true, kPipeMaxThreads, 2>);
+  }
+  return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, false, kPipeMaxThreads, 2>)
+              : reinterpret_cast<const void*>(&encode_pipe_kernel<false, false, kPipeMaxThreads, 2>);
 }
 
-cudaError_t encode_pipe_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm) {
+cudaError_t encode_pipe_attrs(bool bf16, bool full, int threads, size_t smem, int* blocks_per_sm) {
   if (threads > kPipeMaxThreads) return cudaErrorInvalidValue;
-  const void* fn = pipe_kernel(bf16);
+  const void* fn = pipe_kernel(bf16, full);
   // the attribute belongs to the kernel on the current device, not to a plan: it only ever grows, so
   // that every plan can launch
   static std::mutex mu;
-  static size_t granted[kMaxDevices][2] = {};
+  static size_t granted[kMaxDevices][2][2] = {};
   {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(mu);
-    if (smem > granted[dev][bf16 ? 1 : 0]) {
+    if (smem > granted[dev][bf16 ? 1 : 0][full ? 1 : 0]) {
       e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      granted[dev][bf16 ? 1 : 0] = smem;
+      granted[dev][bf16 ? 1 : 0][full ? 1 : 0] = smem;
     }
   }
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads, smem);
 }
 
-cudaError_t launch_encode_pipe(const EncodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream) {
+cudaError_t launch_encode_pipe(const EncodeParams& p, bool full, int grid, int threads, size_t smem, cudaStream_t stream) {
   if (threads > kPipeMaxThreads) return cudaErrorInvalidValue;
-  if (p.dtype == TSQ_BF16) {
-    encode_pipe_kernel<true, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
+  const bool bf16 = p.dtype == TSQ_BF16;
+  if (full) {
+    if (bf16) {
+      encode_pipe_kernel<true, true, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
+    } else {
+      encode_pipe_kernel<false, true, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
+    }
+  } else if (bf16) {
+    encode_pipe_kernel<true, false, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
   } else {
-    encode_pipe_kernel<false, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
+    encode_pipe_kernel<false, false, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
   }
   return cudaGetLastError();
 }

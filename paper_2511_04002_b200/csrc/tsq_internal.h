@@ -103,8 +103,8 @@ struct DecodeParams {
 };
 
 cudaError_t launch_encode_rows(const EncodeParams& p, int grid, int threads, int groups_per_thread, cudaStream_t stream);
-cudaError_t launch_encode_pipe(const EncodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
-cudaError_t encode_pipe_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm);
+cudaError_t launch_encode_pipe(const EncodeParams& p, bool full, int grid, int threads, size_t smem, cudaStream_t stream);
+cudaError_t encode_pipe_attrs(bool bf16, bool full, int threads, size_t smem, int* blocks_per_sm);
 cudaError_t launch_decode(const DecodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
 cudaError_t decode_kernel_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm);
 size_t decode_smem_bytes(uint32_t row_bytes);
