@@ -853,9 +853,9 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         const uint32_t tile_prev = m.tile;
         const uint4* xp = xpark + (n % 3u) * (p.park_stride / 16u);
         uint32_t r[8];
-        Level best = m.lv[p.n_bits - 1];
+        int best_ci = p.n_bits - 1;  // the chosen candidate: its level is read again where it is needed
         int bstar = bmax;
-        const Level top = best;
+        const Level top = m.lv[p.n_bits - 1];
         if (divide) {
           // ---- a row whose scale or zero-point is outside the range of the FMA quotient and of the packed
           //      integer steps (rare): Algorithm 1 with the division instruction, in loops that are not unrolled ----
@@ -868,9 +868,9 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             compute_barrier(nt);
             if (m.S[ci] > p.s_max) break;  // keep the last level that passed
             bstar = p.bits[ci];
-            best = low;
+            best_ci = ci;
           }
-          const Planes8 pl = rolled_pack<BF16>(xw, nt, u, best);
+          const Planes8 pl = rolled_pack<BF16>(xw, nt, u, m.lv[best_ci]);
 #pragma unroll
           for (int k = 0; k < 8; ++k) r[k] = pl.v[k];
         } else {
@@ -894,7 +894,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             compute_barrier(nt);
             if (m.S[ci] > p.s_max) break;  // keep the last level that passed
             bstar = p.bits[ci];
-            best = low;
+            best_ci = ci;
           }
           if (p.n_bits > 1 && bstar == bmax) {
             planes_of_bytes(b2, r);
@@ -909,6 +909,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
               y[4 * j + 2] = c.z;
               y[4 * j + 3] = c.w;
             }
+            const Level best = m.lv[best_ci];
             pack_group<BF16, false>(y, best, r);
           }
         }
@@ -919,8 +920,8 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           publish_aggregate(p, gen4, tile_prev, agg_w, row_cnt);
           m.bstar = static_cast<uint32_t>(bstar);
           m.agg_w = agg_w;
-          m.scale = best.s;
-          m.zp = best.zp;
+          m.scale = m.lv[best_ci].s;
+          m.zp = m.lv[best_ci].zp;
         }
         // ---- planes of the chosen level into the row's slot, in blob order ----
         if (FULL || u < p.units) store_planes(planes + slot * (p.planes_stride / 4u) + u * static_cast<uint32_t>(bstar), r, bstar, true);
