@@ -150,18 +150,20 @@ __device__ __forceinline__ uint32_t split_group(uint32_t (&x)[16], uint32_t nval
 }
 
 // Pass B on one group: sum |(q0 >> sh) - q| over its 32 elements (Algorithm 1's distortion numerator).
+// The codes of two pairs are packed into four bytes, shifted and masked four at a time, and summed by the
+// byte-wise sum-of-absolute-differences instruction: 5 integer instructions per four elements.
 template <bool BF16, bool DIVIDE>
 __device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], const Level& top, const Level& low,
                                                      int sh) {
-  const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
-  uint32_t S2 = 0;  // two 16-bit partial sums: at most 16 * 127 each
+  const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+  uint32_t S = 0;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const uint32_t a = (codes2<BF16, DIVIDE>(x[i], top) >> sh) & shmask;
-    const uint32_t q = codes2<BF16, DIVIDE>(x[i], low);
-    S2 += max_s16x2(a, q) - min_s16x2(a, q);
+  for (int i = 0; i < 16; i += 2) {
+    const uint32_t ct4 = __byte_perm(codes2<BF16, DIVIDE>(x[i], top), codes2<BF16, DIVIDE>(x[i + 1], top), 0x6420);
+    const uint32_t q4 = __byte_perm(codes2<BF16, DIVIDE>(x[i], low), codes2<BF16, DIVIDE>(x[i + 1], low), 0x6420);
+    S = __vsadu4((ct4 >> sh) & shmask, q4) + S;
   }
-  return (S2 & 0xffffu) + (S2 >> 16);
+  return S;
 }
 
 // Pass B for the first lower candidate, keeping what pass C needs if that candidate fails: on return
@@ -169,17 +171,17 @@ __device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], co
 template <bool BF16, bool DIVIDE>
 __device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], const Level& top, const Level& low, int sh,
                                                      uint32_t (&b2)[16]) {
-  const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
-  uint32_t S2 = 0;
+  const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+  uint32_t S = 0;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const uint32_t ct = codes2<BF16, DIVIDE>(x[i], top);
-    const uint32_t a = (ct >> sh) & shmask;
-    const uint32_t q = codes2<BF16, DIVIDE>(x[i], low);
-    S2 += max_s16x2(a, q) - min_s16x2(a, q);
-    b2[i] = ct | ((x[i] >> 8) & 0x00800080u);
+  for (int i = 0; i < 16; i += 2) {
+    const uint32_t ct0 = codes2<BF16, DIVIDE>(x[i], top), ct1 = codes2<BF16, DIVIDE>(x[i + 1], top);
+    const uint32_t q4 = __byte_perm(codes2<BF16, DIVIDE>(x[i], low), codes2<BF16, DIVIDE>(x[i + 1], low), 0x6420);
+    S = __vsadu4((__byte_perm(ct0, ct1, 0x6420) >> sh) & shmask, q4) + S;
+    b2[i] = ct0 | ((x[i] >> 8) & 0x00800080u);
+    b2[i + 1] = ct1 | ((x[i + 1] >> 8) & 0x00800080u);
   }
-  return (S2 & 0xffffu) + (S2 >> 16);
+  return S;
 }
 
 // Bytes of one group (b2[4j + i]: elements 8j + 2i in byte 0 and 8j + 2i + 1 in byte 2) -> bit-planes:
