@@ -56,9 +56,9 @@ __global__ void k_pass_b(const uint4* in, uint32_t* out, float mmax) {
   const Level top = make_level(0.f, mmax, 8), low = make_level(0.f, mmax, 4);
   for (int it = 0; it < kIters; ++it) {
     acc ^= refresh(x);
-    uint32_t b2[16];
-    acc += distortion_first<true, false>(x, top, low, 4, b2);
-    for (int i = 0; i < 16; ++i) acc ^= b2[i];
+    uint32_t tb[8];
+    acc += distortion_first<true, false>(x, top, low, 4, tb);
+    for (int i = 0; i < 8; ++i) acc ^= tb[i];
   }
   out[blockIdx.x * blockDim.x + threadIdx.x] = acc;
 }
@@ -68,9 +68,9 @@ __global__ void k_pass_b_c(const uint4* in, uint32_t* out, float mmax) {
   const Level top = make_level(0.f, mmax, 8), low = make_level(0.f, mmax, 4);
   for (int it = 0; it < kIters; ++it) {
     acc ^= refresh(x);
-    uint32_t b2[16], r[8];
-    acc += distortion_first<true, false>(x, top, low, 4, b2);
-    planes_of_bytes(b2, r);
+    uint32_t tb[8], r[8];
+    acc += distortion_first<true, false>(x, top, low, 4, tb);
+    planes_of_bytes(tb, r);
     for (int i = 0; i < 8; ++i) acc ^= r[i];
   }
   out[blockIdx.x * blockDim.x + threadIdx.x] = acc;

@@ -167,32 +167,35 @@ __device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], co
 }
 
 // Pass B for the first lower candidate, keeping what pass C needs if that candidate fails: on return
-// b2[i] holds the top-level bytes (code | sign << 7) of pair i, low element in byte 0, high in byte 2.
+// tb[i] (i < 4) holds the top-level bytes (code | sign << 7) of elements 2i, 2i + 1, 8 + 2i, 8 + 2i + 1 and
+// tb[4 + i] those of the elements 16 further on.  (Any grouping of four serves the sum; this one is the
+// grouping from which two byte permutes per i give the input of the bit transpose.)
 template <bool BF16, bool DIVIDE>
 __device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], const Level& top, const Level& low, int sh,
-                                                     uint32_t (&b2)[16]) {
+                                                     uint32_t (&tb)[8]) {
   const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
   uint32_t S = 0;
 #pragma unroll
-  for (int i = 0; i < 16; i += 2) {
-    const uint32_t ct0 = codes2<BF16, DIVIDE>(x[i], top), ct1 = codes2<BF16, DIVIDE>(x[i + 1], top);
-    const uint32_t q4 = __byte_perm(codes2<BF16, DIVIDE>(x[i], low), codes2<BF16, DIVIDE>(x[i + 1], low), 0x6420);
-    S = __vsadu4((__byte_perm(ct0, ct1, 0x6420) >> sh) & shmask, q4) + S;
-    b2[i] = ct0 | ((x[i] >> 8) & 0x00800080u);
-    b2[i + 1] = ct1 | ((x[i + 1] >> 8) & 0x00800080u);
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t xa = x[8 * h + i], xb = x[8 * h + 4 + i];  // pairs i of chunks 2h and 2h + 1
+      const uint32_t ct4 = __byte_perm(codes2<BF16, DIVIDE>(xa, top), codes2<BF16, DIVIDE>(xb, top), 0x6420);
+      const uint32_t q4 = __byte_perm(codes2<BF16, DIVIDE>(xa, low), codes2<BF16, DIVIDE>(xb, low), 0x6420);
+      S = __vsadu4((ct4 >> sh) & shmask, q4) + S;
+      tb[4 * h + i] = ct4 | (__byte_perm(xa, xb, 0x7531) & 0x80808080u);  // the sign bits sit in bytes 1 and 3 of a pair
+    }
   }
   return S;
 }
 
-// Bytes of one group (b2[4j + i]: elements 8j + 2i in byte 0 and 8j + 2i + 1 in byte 2) -> bit-planes:
-// on return r[k] = bit k of every byte, k < 7 code bits, k = 7 signs.
-__device__ __forceinline__ void planes_of_bytes(const uint32_t (&b2)[16], uint32_t (&r)[8]) {
+// Bytes of one group as distortion_first leaves them -> bit-planes: on return r[k] = bit k of every byte,
+// k < 7 code bits, k = 7 signs.
+__device__ __forceinline__ void planes_of_bytes(const uint32_t (&tb)[8], uint32_t (&r)[8]) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const uint32_t e = mad_u32(b2[4 + i], 256u, b2[i]);       // bytes: elements 2i, 8 + 2i, 2i + 1, 8 + 2i + 1
-    const uint32_t f = mad_u32(b2[12 + i], 256u, b2[8 + i]);  // the same, 16 further on
-    r[2 * i] = __byte_perm(e, f, 0x5410);              // byte c = element 8c + 2i
-    r[2 * i + 1] = __byte_perm(e, f, 0x7632);          // byte c = element 8c + 2i + 1
+    r[2 * i] = __byte_perm(tb[i], tb[4 + i], 0x6420);      // byte c = element 8c + 2i
+    r[2 * i + 1] = __byte_perm(tb[i], tb[4 + i], 0x7531);  // byte c = element 8c + 2i + 1
   }
   transpose8x32(r);
 }
@@ -878,7 +881,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         } else {
           // ---- Algorithm 1, one candidate per turn; every turn also forms the top-level bytes, which
           //      pass C takes over when the first lower candidate fails (the usual case) ----
-          uint32_t b2[16];
+          uint32_t tb[8];
           for (int ci = p.n_bits - 2; ci >= 0; --ci) {
             uint32_t y[16];
 #pragma unroll
@@ -890,7 +893,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
               y[4 * j + 3] = c.w;
             }
             const Level low = m.lv[ci];
-            uint32_t S = distortion_first<BF16, false>(y, top, low, bmax - p.bits[ci], b2);
+            uint32_t S = distortion_first<BF16, false>(y, top, low, bmax - p.bits[ci], tb);
             S = __reduce_add_sync(kFull, S);
             if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
             compute_barrier(nt);
@@ -899,7 +902,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             best_ci = ci;
           }
           if (p.n_bits > 1 && bstar == bmax) {
-            planes_of_bytes(b2, r);
+            planes_of_bytes(tb, r);
           } else {
             // a lower level was chosen (or there is one candidate only): the parked row once more
             uint32_t y[16];
