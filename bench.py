@@ -44,10 +44,10 @@ FALLBACK_HBM_GBS = 6650.0
 # under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
 # (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
 NCU_TRAFFIC = {
-    "encode": {"sha256": "3450ee45b9461d6379551de2741a58b9f554c33b715037b325203cd8ad733b22",
-               "bytes_per_token": (134338560 + 37416192) / 8192, "hidden": 8192, "dtype": "bf16"},
+    "encode": {"sha256": "ea903a99c029b6df93dd9edf6475b8d32a37f9f29dda51fc30703c64f1c25451",
+               "bytes_per_token": (134309120 + 36406016) / 8192, "hidden": 8192, "dtype": "bf16"},
     "decode": {"sha256": "be5a19566be9449ea9a692b638af3c35bae99b39688b20c4117b9328b6eaedf3",
-               "bytes_per_token": (68643840 + 77444608) / 8192, "hidden": 8192, "dtype": "bf16"},
+               "bytes_per_token": (68643584 + 76800512) / 8192, "hidden": 8192, "dtype": "bf16"},
 }
 KERNEL_NAMES = {"encode": "encode_pipe_kernel (encode_rows_kernel for few or very long rows)", "decode": "decode_kernel"}
 
