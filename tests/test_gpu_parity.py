@@ -74,6 +74,27 @@ def test_many_rows_some_needing_the_division_instruction(dtype, shape, delta):
     full_parity(x.to(dtype).contiguous(), INF, [2, 3, 4, 8], delta, check_cross=False)
 
 
+@pytest.mark.parametrize("case", range(24))
+def test_randomized_many_row_cases(case):
+    # seeded draws over the shapes, candidate sets, thresholds and tolerances that select between the kernels
+    # and between their paths (whole and ragged groups, descent depth, outlier lists that overflow)
+    rng = np.random.default_rng(1000 + case)
+    H = int(rng.choice([8, 72, 264, 1024, 2048, 4096, 4104, 5120, 8192, 8184])) if rng.random() < 0.7 else int(rng.integers(1, 1025)) * 8
+    T = int(rng.integers(297, 1400))
+    if T * H > 6_000_000:
+        T = max(297, 6_000_000 // H)
+    dtype = torch.float16 if rng.random() < 0.5 else torch.bfloat16
+    g = torch.Generator().manual_seed(int(rng.integers(1 << 30)))
+    scale = float(rng.choice([0.3, 1.0, 2.0, 5.0]))
+    v = torch.randn((T, H), generator=g) * scale * torch.exp(torch.randn((T, 1), generator=g) * 0.5)
+    if rng.random() < 0.5:
+        v = torch.where(torch.rand((T, H), generator=g) < 0.01, v * 30, v)
+    bits = [[2, 4, 8], [2, 3, 4, 8], [8], [3, 5], [2, 3, 4, 5, 6, 7, 8]][int(rng.integers(5))]
+    delta = float(rng.choice([0.2, 0.0, 0.5, 1e9, -1.0]))
+    tau = float(rng.choice([6.0, 1.0, 3.0, INF]))
+    full_parity(v.to(dtype).contiguous(), tau, bits, delta, check_cross=False)
+
+
 @pytest.mark.parametrize("hidden", [16384, 65536])
 def test_long_rows(hidden):
     x = rand16((5, hidden), torch.bfloat16, seed=hidden, scale=1.5, outlier_rate=0.001)
