@@ -44,7 +44,7 @@ FALLBACK_HBM_GBS = 6650.0
 # under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
 # (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
 NCU_TRAFFIC = {
-    "encode": {"sha256": "ea903a99c029b6df93dd9edf6475b8d32a37f9f29dda51fc30703c64f1c25451",
+    "encode": {"sha256": "8ae22dc679f0978b8b718c7aae6638725c337f3b19467d8168abc830ebfabaf8",
                "bytes_per_token": (134309120 + 36406016) / 8192, "hidden": 8192, "dtype": "bf16"},
     "decode": {"sha256": "be5a19566be9449ea9a692b638af3c35bae99b39688b20c4117b9328b6eaedf3",
                "bytes_per_token": (68643584 + 76800512) / 8192, "hidden": 8192, "dtype": "bf16"},

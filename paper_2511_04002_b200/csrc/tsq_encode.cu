@@ -28,15 +28,17 @@
 //                       that pass B already formed.
 //
 // The binding resource is the integer / logic pipe, which issues at half the rate of the FMA pipe:
-// the passes work on two 16-bit elements per 32-bit register wherever they can, and shifts and
-// byte merges are written as integer multiply-adds so that they go to the FMA pipe instead.
+// the passes work on two 16-bit elements per 32-bit register wherever they can (four codes as bytes
+// in the distortion sum and on the way to the bit transpose), and some shifts and merges are written
+// as integer multiply-adds so that they go to the FMA pipe instead.
 //
 // Variable-length placement: where a token's planes and CSR entries start is an exclusive prefix
 // sum over all earlier tokens.  It is resolved with a decoupled look-back over per-token
 // descriptors in the workspace.  Rows are numbered by an atomic ticket taken by a running CTA,
 // so a row only ever waits for rows whose CTAs are already running, and a row publishes its own
 // sizes before it waits for anything.  A look-back step reads 256 descriptor pairs at once (eight
-// independent loads per lane).  Every wait is bounded and fails into a status word.
+// independent loads per lane) in the one-CTA-per-row kernel and 32 in the pipelined kernel.  Every wait
+// is bounded and fails into a status word.
 //
 // Arithmetic contract: the codes equal  clamp(rint(m / s) - zp, 0, Qmax)  with the IEEE binary32
 // quotient m / s.  The quotient is formed without the division instruction: r = fl(1 / s) once per
