@@ -56,8 +56,8 @@ __global__ void k_pass_b(const uint4* in, uint32_t* out, float mmax) {
   const Level top = make_level(0.f, mmax, 8), low = make_level(0.f, mmax, 4);
   for (int it = 0; it < kIters; ++it) {
     acc ^= refresh(x);
-    uint32_t tb[8];
-    acc += distortion_first<true, false>(x, top, low, 4, tb);
+    uint32_t tb[8], ql[8];
+    acc += distortion_first<true, false>(x, top, low, 4, tb, ql);
     for (int i = 0; i < 8; ++i) acc ^= tb[i];
   }
   out[blockIdx.x * blockDim.x + threadIdx.x] = acc;
@@ -68,8 +68,8 @@ __global__ void k_pass_b_c(const uint4* in, uint32_t* out, float mmax) {
   const Level top = make_level(0.f, mmax, 8), low = make_level(0.f, mmax, 4);
   for (int it = 0; it < kIters; ++it) {
     acc ^= refresh(x);
-    uint32_t tb[8], r[8];
-    acc += distortion_first<true, false>(x, top, low, 4, tb);
+    uint32_t tb[8], ql[8], r[8];
+    acc += distortion_first<true, false>(x, top, low, 4, tb, ql);
     planes_of_bytes(tb, r);
     for (int i = 0; i < 8; ++i) acc ^= r[i];
   }

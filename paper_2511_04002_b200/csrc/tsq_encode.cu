@@ -174,7 +174,7 @@ __device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], co
 // grouping from which two byte permutes per i give the input of the bit transpose.)
 template <bool BF16, bool DIVIDE>
 __device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], const Level& top, const Level& low, int sh,
-                                                     uint32_t (&tb)[8]) {
+                                                     uint32_t (&tb)[8], uint32_t (&ql)[8]) {
   const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
   uint32_t S = 0;
 #pragma unroll
@@ -186,6 +186,27 @@ __device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], co
       const uint32_t q4 = __byte_perm(codes2<BF16, DIVIDE>(xa, low), codes2<BF16, DIVIDE>(xb, low), 0x6420);
       S = __vsadu4((ct4 >> sh) & shmask, q4) + S;
       tb[4 * h + i] = ct4 | (__byte_perm(xa, xb, 0x7531) & 0x80808080u);  // the sign bits sit in bytes 1 and 3 of a pair
+      ql[4 * h + i] = q4;  // the candidate's own codes, same grouping, no signs: its planes if it is the one chosen
+    }
+  }
+  return S;
+}
+
+// Pass B for a further candidate: the top-level codes come from the bytes the first turn left.
+template <bool BF16>
+__device__ __forceinline__ uint32_t distortion_next(const uint32_t (&x)[16], const uint32_t (&tb)[8], const Level& low, int sh,
+                                                    uint32_t (&ql)[8]) {
+  // a byte of tb is code | sign << 7: shifted right by sh >= 1, the sign bit and the bits that come in from
+  // the next byte all land above the mask
+  const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+  uint32_t S = 0;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t q4 = __byte_perm(codes2<BF16, false>(x[8 * h + i], low), codes2<BF16, false>(x[8 * h + 4 + i], low), 0x6420);
+      S = __vsadu4((tb[4 * h + i] >> sh) & shmask, q4) + S;
+      ql[4 * h + i] = q4;
     }
   }
   return S;
@@ -881,10 +902,13 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
 #pragma unroll
           for (int k = 0; k < 8; ++k) r[k] = pl.v[k];
         } else {
-          // ---- Algorithm 1, one candidate per turn; every turn also forms the top-level bytes, which
-          //      pass C takes over when the first lower candidate fails (the usual case) ----
-          uint32_t tb[8];
-          for (int ci = p.n_bits - 2; ci >= 0; --ci) {
+          // ---- Algorithm 1, one candidate per turn.  The first turn also leaves the top-level bytes (what pass C
+          //      packs when the first lower candidate fails, the usual case, and where later turns take the
+          //      top-level codes from); every turn leaves its candidate's codes, which become the planes when
+          //      that candidate is the last to pass.  With one candidate only, the turn runs for its bytes alone. ----
+          uint32_t tb[8], lb[8];
+          int ci = p.n_bits - 2;
+          {
             uint32_t y[16];
 #pragma unroll
             for (uint32_t j = 0; j < 4; ++j) {
@@ -894,31 +918,48 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
               y[4 * j + 2] = c.z;
               y[4 * j + 3] = c.w;
             }
-            const Level low = m.lv[ci];
-            uint32_t S = distortion_first<BF16, false>(y, top, low, bmax - p.bits[ci], tb);
-            S = __reduce_add_sync(kFull, S);
-            if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
+            const int c0 = ci >= 0 ? ci : 0;
+            const Level low = m.lv[c0];
+            uint32_t S = distortion_first<BF16, false>(y, top, low, bmax - p.bits[c0], tb, lb);
+            if (ci >= 0) {
+              S = __reduce_add_sync(kFull, S);
+              if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
+            }
+          }
+          bool passed = false;
+          if (ci >= 0) {
             compute_barrier(nt);
-            if (m.S[ci] > p.s_max) break;  // keep the last level that passed
+            passed = m.S[ci] <= p.s_max;
+          }
+          if (passed) {
             bstar = p.bits[ci];
             best_ci = ci;
-          }
-          if (p.n_bits > 1 && bstar == bmax) {
-            planes_of_bytes(tb, r);
-          } else {
-            // a lower level was chosen (or there is one candidate only): the parked row once more
-            uint32_t y[16];
+            for (--ci; ci >= 0; --ci) {
+              uint32_t y[16], ql[8];
 #pragma unroll
-            for (uint32_t j = 0; j < 4; ++j) {
-              const uint4 c = xp[park_index(nt, u, j)];
-              y[4 * j + 0] = c.x;
-              y[4 * j + 1] = c.y;
-              y[4 * j + 2] = c.z;
-              y[4 * j + 3] = c.w;
+              for (uint32_t j = 0; j < 4; ++j) {
+                const uint4 c = xp[park_index(nt, u, j)];
+                y[4 * j + 0] = c.x;
+                y[4 * j + 1] = c.y;
+                y[4 * j + 2] = c.z;
+                y[4 * j + 3] = c.w;
+              }
+              const Level low = m.lv[ci];
+              uint32_t S = distortion_next<BF16>(y, tb, low, bmax - p.bits[ci], ql);
+              S = __reduce_add_sync(kFull, S);
+              if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
+              compute_barrier(nt);
+              if (m.S[ci] > p.s_max) break;  // keep the last level that passed
+              bstar = p.bits[ci];
+              best_ci = ci;
+#pragma unroll
+              for (int k = 0; k < 8; ++k) lb[k] = ql[k];
             }
-            const Level best = m.lv[best_ci];
-            pack_group<BF16, false>(y, best, r);
+            // the chosen candidate's codes with the signs of the top-level bytes
+#pragma unroll
+            for (int k = 0; k < 8; ++k) tb[k] = lb[k] | (tb[k] & 0x80808080u);
           }
+          planes_of_bytes(tb, r);
         }
         const uint32_t row_cnt = m.row_cnt;
         const uint32_t agg_w = static_cast<uint32_t>(bstar) * p.lay.wpp;
