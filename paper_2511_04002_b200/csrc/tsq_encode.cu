@@ -856,10 +856,8 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           sh.next_tile[(n_a + 1u) & 1u] = ticket_ahead;
         }
         if (have_prev) {
-          // passes B and C of row n_a - 1 need its levels, and the slot that its planes go to
-          // must have been emptied by the placement of row n_a - 1 - p.ring
+          // pass B of row n_a - 1 needs its levels
           wait_beyond(&sh.lv_ready, n_a - 1u, sh, false, 100u);
-          if (n_a - 1u >= p.ring) wait_beyond(&sh.placed, n_a - 1u - p.ring, sh, false, 100u);
         }
       }
       compute_barrier(nt);
@@ -971,8 +969,13 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           m.scale = m.lv[best_ci].s;
           m.zp = m.lv[best_ci].zp;
         }
+        // ---- the slot that the row's planes and CSR entries go to must have been emptied by the placement of
+        //      row n - p.ring.  Every thread looks for itself, and only now: the row's sizes are published
+        //      already, so a CTA whose ring is full does not keep the rows behind it (in other CTAs) waiting
+        //      for this row's sizes on top of its own wait. ----
+        const bool slot_free = n < p.ring || wait_beyond(&sh.placed, n - p.ring, sh, false, 100u);
         // ---- planes of the chosen level into the row's slot, in blob order ----
-        if (FULL || u < p.units) store_planes(planes + slot * (p.planes_stride / 4u) + u * static_cast<uint32_t>(bstar), r, bstar, true);
+        if (slot_free && (FULL || u < p.units)) store_planes(planes + slot * (p.planes_stride / 4u) + u * static_cast<uint32_t>(bstar), r, bstar, true);
         // ---- CSR entries of T_above into the row's list: ascending columns, original patterns ----
         const uint32_t flagged = __ballot_sync(kFull, cnt_prev != 0u);
         if (flagged != 0u) {
@@ -988,7 +991,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             }
             before = incl - cnt_prev;
           }
-          if (cnt_prev != 0u && row_cnt <= p.csr_cap) {
+          if (slot_free && cnt_prev != 0u && row_cnt <= p.csr_cap) {
             uint32_t* list = csr + slot * p.csr_cap;
             const uint16_t* x16 = p.x + static_cast<size_t>(tile_prev) * p.hidden;
             uint32_t at = m.part.warp_cnt[warp] + before;
