@@ -204,30 +204,46 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
     p->pipe_threads = static_cast<int>(p->pipe_compute) + 64;
     p->pipe_park = p->pipe_compute * 64u;
     p->pipe_planes = (static_cast<uint32_t>(p->bmax) * p->units * 4u + 127u) & ~127u;
-    // a CSR list of two entries per group per ring slot (one outlier in sixteen elements; rows above that
-    // take a slower path)
-    p->pipe_csr_cap = 2u * p->pipe_compute;
-    const auto smem_for = [&](uint32_t ring) {
-      return 3u * static_cast<size_t>(p->pipe_park) + ring * (static_cast<size_t>(p->pipe_planes) + 4u * static_cast<size_t>(p->pipe_csr_cap));
-    };
-    p->pipe_ring = 4u;
-    p->pipe_smem = smem_for(p->pipe_ring);
+    // A CSR list per ring slot: four entries per group (one outlier in eight elements; rows above that take
+    // a slower path that holds up their CTA's placement) when that costs neither a resident CTA nor ring
+    // depth below 6 (or below what two entries per group give), else two entries per group.
     p->pipe_ctas_per_sm = 0;
-    if (ok && p->pipe_threads <= kPipeMaxThreads && p->pipe_smem + 8192 <= static_cast<size_t>(smem_optin)) {
+    p->pipe_ring = 4u;
+    p->pipe_csr_cap = 2u * p->pipe_compute;
+    p->pipe_smem = 0;
+    int base_blocks = 0;
+    uint32_t base_ring = 0;
+    for (uint32_t per_group = 2u; ok && per_group <= 4u && p->pipe_threads <= kPipeMaxThreads; per_group += 2u) {
+      const uint32_t cap = per_group * p->pipe_compute;
+      const auto smem_for = [&](uint32_t ring) {
+        return 3u * static_cast<size_t>(p->pipe_park) + ring * (static_cast<size_t>(p->pipe_planes) + 4u * static_cast<size_t>(cap));
+      };
+      if (smem_for(4u) + 8192 > static_cast<size_t>(smem_optin)) break;
       int blocks = 0;
-      ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, p->pipe_threads, p->pipe_smem, &blocks) == cudaSuccess;
-      p->pipe_ctas_per_sm = blocks;
+      ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, p->pipe_threads, smem_for(4u), &blocks) == cudaSuccess;
+      if (!ok || blocks < 1) break;
       // the deepest ring that leaves the number of resident CTAs as it is
-      for (uint32_t ring = static_cast<uint32_t>(kMaxRing); ok && blocks > 0 && ring > 4u; --ring) {
-        if (smem_for(ring) + 8192 > static_cast<size_t>(smem_optin)) continue;
+      uint32_t ring = 4u;
+      for (uint32_t r = static_cast<uint32_t>(kMaxRing); ok && r > 4u; --r) {
+        if (smem_for(r) + 8192 > static_cast<size_t>(smem_optin)) continue;
         int b = 0;
-        ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, p->pipe_threads, smem_for(ring), &b) == cudaSuccess;
+        ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, p->pipe_threads, smem_for(r), &b) == cudaSuccess;
         if (ok && b == blocks) {
-          p->pipe_ring = ring;
-          p->pipe_smem = smem_for(ring);
+          ring = r;
           break;
         }
       }
+      if (!ok) break;
+      if (per_group == 2u) {
+        base_blocks = blocks;
+        base_ring = ring;
+      } else if (blocks != base_blocks || ring < (base_ring < 6u ? base_ring : 6u)) {
+        break;  // the longer lists cost too much: keep the shorter ones
+      }
+      p->pipe_ctas_per_sm = blocks;
+      p->pipe_ring = ring;
+      p->pipe_csr_cap = cap;
+      p->pipe_smem = smem_for(ring);
     }
   }
   cudaSetDevice(prev_dev);
