@@ -924,6 +924,9 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
               if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
             }
           }
+          // pass C at the top level right away: the usual outcome, and work to do while the other warps
+          // arrive at the barrier (a row that goes lower transposes once more, below)
+          planes_of_bytes(tb, r);
           bool passed = false;
           if (ci >= 0) {
             compute_barrier(nt);
@@ -956,8 +959,8 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             // the chosen candidate's codes with the signs of the top-level bytes
 #pragma unroll
             for (int k = 0; k < 8; ++k) tb[k] = lb[k] | (tb[k] & 0x80808080u);
+            planes_of_bytes(tb, r);
           }
-          planes_of_bytes(tb, r);
         }
         const uint32_t row_cnt = m.row_cnt;
         const uint32_t agg_w = static_cast<uint32_t>(bstar) * p.lay.wpp;
