@@ -44,10 +44,10 @@ FALLBACK_HBM_GBS = 6650.0
 # under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
 # (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
 NCU_TRAFFIC = {
-    "encode": {"sha256": "429e8fb5aef789cca4971619bb7ca4ee359a78f8deddb645a504c4c6642c2ddc",
-               "bytes_per_token": (134301952 + 35568640) / 8192, "hidden": 8192, "dtype": "bf16"},
+    "encode": {"sha256": "5a0390c1cf5272d29e24e491a6bee0f682506c09c2b85718488170b4243e25a7",
+               "bytes_per_token": (134295296 + 35242240) / 8192, "hidden": 8192, "dtype": "bf16"},
     "decode": {"sha256": "be5a19566be9449ea9a692b638af3c35bae99b39688b20c4117b9328b6eaedf3",
-               "bytes_per_token": (68645888 + 77188352) / 8192, "hidden": 8192, "dtype": "bf16"},
+               "bytes_per_token": (68644352 + 77484800) / 8192, "hidden": 8192, "dtype": "bf16"},
 }
 KERNEL_NAMES = {"encode": "encode_pipe_kernel (encode_rows_kernel for few or very long rows)", "decode": "decode_kernel"}
 
