@@ -44,7 +44,7 @@ FALLBACK_HBM_GBS = 6650.0
 # under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
 # (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
 NCU_TRAFFIC = {
-    "encode": {"sha256": "5a0390c1cf5272d29e24e491a6bee0f682506c09c2b85718488170b4243e25a7",
+    "encode": {"sha256": "0a591ccb46927174d99eaa8f9cda8910c211a22fb49172334b0170361d2e7c87",
                "bytes_per_token": (134319104 + 36340480) / 8192, "hidden": 8192, "dtype": "bf16"},
     "decode": {"sha256": "be5a19566be9449ea9a692b638af3c35bae99b39688b20c4117b9328b6eaedf3",
                "bytes_per_token": (68642816 + 76561408) / 8192, "hidden": 8192, "dtype": "bf16"},
