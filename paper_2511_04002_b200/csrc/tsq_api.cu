@@ -284,14 +284,23 @@ tsq_status_t tsq_workspace_init(const tsq_plan_t* plan, void* ws_dev, size_t ws_
   return cudaGetLastError() == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
 }
 
-tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t tokens, void* blob_dev, size_t blob_bytes,
-                        void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+// Argument checks of an encode call, made before anything is enqueued.
+static tsq_status_t check_encode_args(const tsq_plan_t* plan, const void* x_dev, int64_t tokens, const void* blob_dev,
+                                      size_t blob_bytes, const void* ws_dev, size_t ws_bytes) {
   if (!plan || !blob_dev || !ws_dev || tokens < 0 || static_cast<unsigned long long>(tokens) > plan->max_tokens)
     return TSQ_ERR_INVALID_ARG;
   if (tokens > 0 && !x_dev) return TSQ_ERR_INVALID_ARG;
   if (!aligned16(x_dev) || !aligned16(blob_dev) || !aligned16(ws_dev)) return TSQ_ERR_INVALID_ARG;
   const BlobLayout L = layout_for(plan, static_cast<unsigned long long>(tokens));
   if (blob_bytes < L.total || ws_bytes < plan->workspace_bytes) return TSQ_ERR_BUFFER_TOO_SMALL;
+  return TSQ_OK;
+}
+
+tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t tokens, void* blob_dev, size_t blob_bytes,
+                        void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  const tsq_status_t args_ok = check_encode_args(plan, x_dev, tokens, blob_dev, blob_bytes, ws_dev, ws_bytes);
+  if (args_ok != TSQ_OK) return args_ok;
+  const BlobLayout L = layout_for(plan, static_cast<unsigned long long>(tokens));
 
   EncodeParams p;
   std::memset(&p, 0, sizeof p);
@@ -368,12 +377,24 @@ tsq_status_t tsq_encode_noalloc(const tsq_plan_t* plan, const void* x_dev, int64
                                 size_t blob_bytes, void* cuda_stream) {
   if (!plan) return TSQ_ERR_INVALID_ARG;
   if (plan->max_tokens > kStaticMaxTokens || plan->workspace_bytes > kStaticWsBytes) return TSQ_ERR_UNSUPPORTED;
+  // the stream (and the kernels launched on it) belong to the current device: it has to be the plan's
+  int current = -1;
+  if (cudaGetDevice(&current) != cudaSuccess) {
+    cudaGetLastError();
+    return TSQ_ERR_CUDA;
+  }
+  if (current != plan->device) return TSQ_ERR_INVALID_ARG;
   void* ws = nullptr;
   if (static_workspace(plan->device, &ws) != cudaSuccess) {
     cudaGetLastError();
     return TSQ_ERR_CUDA;
   }
-  // the array keeps whatever the last call left (including an unfinished call's tickets): start clean
+  // every argument error is reported before the shared array is touched
+  const tsq_status_t args_ok = check_encode_args(plan, x_dev, tokens, blob_dev, blob_bytes, ws, kStaticWsBytes);
+  if (args_ok != TSQ_OK) return args_ok;
+  // The array keeps whatever the last call left (including an unfinished call's tickets): start clean.
+  // This also zeroes the generation counter and the recorded capacity: every call through this entry
+  // point runs as generation 1, so the wrap-around path that reads the capacity is never taken here.
   if (cudaMemsetAsync(ws, 0, plan->workspace_bytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
     cudaGetLastError();
     return TSQ_ERR_CUDA;

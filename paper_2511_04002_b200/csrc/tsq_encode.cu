@@ -499,6 +499,10 @@ __device__ void finish_call(const EncodeParams& p, uint32_t gen4) {
   }
   write_header(p, tw, to);
   reinterpret_cast<BlobHeader*>(p.blob)->status = e;
+  if (p.tokens == 0u) {  // no row writes the leading zeros of the two prefix-sum sections
+    reinterpret_cast<uint32_t*>(p.blob + p.lay.off_word_off)[0] = 0u;
+    reinterpret_cast<uint32_t*>(p.blob + p.lay.off_out_ptr)[0] = 0u;
+  }
   if (e != 0u) atomicCAS(&p.ws->enc_status, 0u, e);
   uint32_t g = (gen4 >> 2);
   if (g >= kGenWrap) {
