@@ -112,6 +112,18 @@ tsq_status_t tsq_plan_sizes(const tsq_plan_t *plan, int64_t tokens, tsq_sizes_t 
 tsq_status_t tsq_workspace_init(const tsq_plan_t *plan, void *ws_dev, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Set how long the encoder's device-side waits may last before they give up with TSQ_ERR_TIMEOUT.  The
+ * only such wait is the placement look-back: a row's offsets are the prefix sums over every earlier
+ * row, and a row polls the workspace until those rows have published theirs.  `polls` counts polls of
+ * one descriptor (200 ns apart for the first 32, then 1 us apart); 0 restores the built-in limit of
+ * 2^20 polls (about one second), which is also what tsq_workspace_init sets.  A wait can only run out
+ * when the workspace was not initialised, is shared by calls that overlap on the GPU, or was
+ * overwritten: the limit exists so that such a mistake ends in a status instead of a hang.  The
+ * setting is kept in the workspace (DEVICE) and is written on `cuda_stream`.
+ */
+tsq_status_t tsq_workspace_set_wait_limit(void *ws_dev, uint32_t polls, void *cuda_stream);
+
+/*
  * Encode x (DEVICE, [tokens x hidden]) into blob (DEVICE, >= blob_bytes from tsq_plan_sizes,
  * 16-byte aligned): TS (Eq. "ts") + TAB-Q (Algorithm 1, token-wise) + bit-plane packing, one
  * kernel launch.  tokens == 0 writes an empty, valid blob.  Returns argument errors before

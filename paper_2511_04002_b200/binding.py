@@ -16,7 +16,7 @@ F16, BF16 = 0, 1
 STATUS = {0: "TSQ_OK", 1: "TSQ_ERR_INVALID_ARG", 2: "TSQ_ERR_UNSUPPORTED", 3: "TSQ_ERR_BUFFER_TOO_SMALL",
           4: "TSQ_ERR_CUDA", 5: "TSQ_ERR_CORRUPT_BLOB", 6: "TSQ_ERR_OUTLIER_OVERFLOW", 7: "TSQ_ERR_TIMEOUT"}
 
-EXPORTS = ["tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_encode", "tsq_encode_noalloc", "tsq_decode",
+EXPORTS = ["tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_workspace_set_wait_limit", "tsq_encode", "tsq_encode_noalloc", "tsq_decode",
            "tsq_blob_info",
            "tsq_workspace_status", "tsq_encode_host", "tsq_decode_host", "tsq_kernel_launch_count",
            "tsq_plan_destroy", "tsq_status_string"]
@@ -54,6 +54,7 @@ def lib() -> C.CDLL:
                            C.c_int32, C.c_float, i64]
     L.tsq_plan_sizes.argtypes = [vp, i64, C.POINTER(_Sizes)]
     L.tsq_workspace_init.argtypes = [vp, vp, sz, vp]
+    L.tsq_workspace_set_wait_limit.argtypes = [vp, C.c_uint32, vp]
     L.tsq_encode.argtypes = [vp, vp, i64, vp, sz, vp, sz, vp]
     L.tsq_encode_noalloc.argtypes = [vp, vp, i64, vp, sz, vp]
     L.tsq_encode_noalloc.restype = C.c_int
@@ -62,7 +63,7 @@ def lib() -> C.CDLL:
     L.tsq_workspace_status.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), vp]
     L.tsq_encode_host.argtypes = [vp, vp, i64, vp, sz, C.POINTER(C.c_uint64), vp, vp, vp, sz, vp]
     L.tsq_decode_host.argtypes = [vp, vp, sz, i64, vp, vp, vp, vp, sz, vp]
-    for name in ("tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_encode", "tsq_decode", "tsq_blob_info",
+    for name in ("tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_workspace_set_wait_limit", "tsq_encode", "tsq_decode", "tsq_blob_info",
                  "tsq_workspace_status", "tsq_encode_host", "tsq_decode_host"):
         getattr(L, name).restype = C.c_int
     L.tsq_kernel_launch_count.argtypes = []
@@ -140,6 +141,9 @@ class Plan:
 
     def workspace_init(self, ws: torch.Tensor, stream=None) -> None:
         _check(lib().tsq_workspace_init(self._h, ws.data_ptr(), ws.numel(), _stream(stream)), "tsq_workspace_init")
+
+    def workspace_set_wait_limit(self, ws: torch.Tensor, polls: int, stream=None) -> None:
+        _check(lib().tsq_workspace_set_wait_limit(ws.data_ptr(), polls, _stream(stream)), "tsq_workspace_set_wait_limit")
 
     def encode(self, x: torch.Tensor, blob: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
         assert x.is_cuda and x.is_contiguous() and x.dtype == self.dtype and x.dim() == 2 and x.shape[1] == self.hidden

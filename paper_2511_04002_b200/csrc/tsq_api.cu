@@ -79,6 +79,7 @@ cudaError_t static_workspace(int device, void** out) {
 }
 
 __global__ void workspace_init_kernel(WsControl* ws, uint32_t desc_capacity) { ws->desc_capacity = desc_capacity; }
+__global__ void workspace_wait_limit_kernel(WsControl* ws, uint32_t polls) { ws->poll_limit = polls; }
 
 }  // namespace
 }  // namespace tsq
@@ -280,6 +281,13 @@ tsq_status_t tsq_workspace_init(const tsq_plan_t* plan, void* ws_dev, size_t ws_
   if (cudaMemsetAsync(ws_dev, 0, plan->workspace_bytes, st) != cudaSuccess) return TSQ_ERR_CUDA;
   const uint32_t cap = static_cast<uint32_t>(plan->max_tokens > 0 ? plan->max_tokens : 1);
   workspace_init_kernel<<<1, 1, 0, st>>>(static_cast<WsControl*>(ws_dev), cap);
+  g_launches.fetch_add(1);
+  return cudaGetLastError() == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
+}
+
+tsq_status_t tsq_workspace_set_wait_limit(void* ws_dev, uint32_t polls, void* cuda_stream) {
+  if (!ws_dev || !aligned16(ws_dev)) return TSQ_ERR_INVALID_ARG;
+  workspace_wait_limit_kernel<<<1, 1, 0, static_cast<cudaStream_t>(cuda_stream)>>>(static_cast<WsControl*>(ws_dev), polls);
   g_launches.fetch_add(1);
   return cudaGetLastError() == cudaSuccess ? TSQ_OK : TSQ_ERR_CUDA;
 }

@@ -181,6 +181,31 @@ __device__ __forceinline__ void transpose8x32(uint32_t (&r)[8]) {
   }
 }
 
+// (a & mask) | (b & ~mask) in one three-input logic instruction
+__device__ __forceinline__ uint32_t bit_select(uint32_t mask, uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("lop3.b32 %0, %1, %2, %3, 0xCA;" : "=r"(r) : "r"(mask), "r"(a), "r"(b));
+  return r;
+}
+
+// The same transpose with each exchange written as two bit selections (a shift and a three-input logic
+// instruction per word, the left shift as a multiplication so that it goes to the FMA pipe) instead of the
+// xor-swap's five instructions.
+__device__ __forceinline__ void transpose8x32_select(uint32_t (&r)[8]) {
+#pragma unroll
+  for (int b = 0; b < 3; ++b) {
+    const int sh = 1 << b;
+    const uint32_t mask_lo = (b == 0) ? 0x55555555u : (b == 1) ? 0x33333333u : 0x0f0f0f0fu;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (i & sh) continue;
+      const uint32_t lo = r[i], hi = r[i | sh];
+      r[i | sh] = bit_select(mask_lo, lo >> sh, hi);
+      r[i] = bit_select(mask_lo, lo, mad_u32(hi, 1u << sh, 0u));
+    }
+  }
+}
+
 }  // namespace tsq
 
 #endif  // TSQ_DEVICE_CUH_

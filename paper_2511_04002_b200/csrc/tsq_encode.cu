@@ -41,14 +41,19 @@
 // is bounded and fails into a status word.
 //
 // Arithmetic contract: the codes equal  clamp(rint(m / s) - zp, 0, Qmax)  with the IEEE binary32
-// quotient m / s.  The quotient is formed without the division instruction: r = fl(1 / s) once per
-// row and level, then per element q0 = fl(m * r), the exact residual m - q0 * s (one FMA) and
-// q = fl(q0 + residual * r).  This is the classical FMA division step: with a correctly rounded
-// reciprocal and no over- or underflow, q is the correctly rounded quotient.  (A single
-// fl(m * r) is not enough: 16-bit inputs put m / s on or next to a rounding boundary k + 1/2 in
-// almost every row, and there the two can round differently.)  rint is one addition of 2^23.  Rows
-// whose scale is so large or so small that an intermediate product could leave the normal range,
-// or whose zero-point does not fit the packed 16-bit integer steps, use the division instruction.
+// quotient m / s.  "Plain" rows (nearly every row of real data: zero-point 0, which any row with an
+// outlier or a tiny element has; no code above Qmax; scale in [2^-60, 2^60], so that no intermediate
+// leaves the normal range) form the quotient without the division instruction: r = fl(1 / s) once
+// per row and level, then per element q0 = fl(m * r), the residual m - q0 * s (one FMA) and
+// q = fl(q0 + residual * r), two elements at a time with the packed binary32 instructions (each
+// lane rounds to nearest even, as the scalar instructions do).  rint is one addition of 2^23, and
+// the code is the low byte of the sum's pattern: no subtraction, no clamp.  What has to hold is
+// that rint(q) equals rint(fl(m / s)) for every 16-bit magnitude m of the row; a host-side test
+// checks the three-operation sequence in exact arithmetic against the true quotient for every
+// 16-bit pattern over many ranges and levels, and the GPU parity tests compare every code.  (A
+// single fl(m * r) is not enough: 16-bit inputs put m / s on or next to a rounding boundary
+// k + 1/2 in almost every row, and there the two can round differently.)  Every other row goes
+// through the division instruction in compact loops.
 
 #include <mutex>
 
@@ -59,20 +64,17 @@ namespace tsq {
 namespace {
 
 constexpr float kRoundMagic = 8388608.0f;  // 2^23: adding it to 0 <= y < 2^23 rounds y to an integer, ties to even
-constexpr uint32_t kRoundMagicHi = 0x4B00u;  // upper 16 bits of the pattern of 2^23
-constexpr uint32_t kLookbackPollLimit = 1u << 20;
-constexpr uint32_t kHandshakePollLimit = 1u << 22;
+constexpr uint32_t kLookbackPollLimit = 1u << 20;  // polls of one descriptor (200 ns to 1 us apart): about a second
+constexpr uint32_t kHandshakeFactor = 4u;          // handshakes inside a CTA poll faster: four times as many polls
 
 // AIQ parameters of one candidate level for one row (Eq. "Proposed").
-struct __align__(16) Level {  // 32 bytes: what the usual path reads comes first, in one 16-byte load
-  float s;       // scale
-  float r;       // fl(1 / s)
-  uint32_t nz2;  // -zp in the low half, -zp - kRoundMagicHi in the high half (see codes2)
-  uint32_t qm2;  // qmax in both 16-bit halves
-  int zp;        // zero-point rint(m_min / s)
-  int qmax;      // 2^(b-1) - 1
-  int packed;    // scale and zero-point in the range where the FMA quotient and the packed steps are safe
-  int pad;
+struct __align__(16) Level {
+  float s;    // scale
+  float r;    // fl(1 / s)
+  int zp;     // zero-point rint(m_min / s)
+  int qmax;   // 2^(b-1) - 1
+  int plain;  // the fast steps apply: FMA quotient safe, zero-point 0, no code needs the clamp (see the file header)
+  int pad[3];
 };
 
 __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
@@ -80,33 +82,88 @@ __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
   c.qmax = (1 << (b - 1)) - 1;
   const float range = __fsub_rn(mmax, mmin);
   c.s = range > 0.0f ? __fdiv_rn(range, static_cast<float>(c.qmax)) : (mmax > 0.0f ? mmax : 1.0f);
-  c.zp = __float2int_rn(__fdiv_rn(mmin, c.s));
+  c.zp = mmin > 0.0f ? __float2int_rn(__fdiv_rn(mmin, c.s)) : 0;  // 0 / s = 0: the usual row needs no division here
   c.r = __frcp_rn(c.s);
-  c.nz2 = (static_cast<uint32_t>(-c.zp) & 0xffffu) | (static_cast<uint32_t>(-c.zp - static_cast<int>(kRoundMagicHi)) << 16);
-  c.qm2 = static_cast<uint32_t>(c.qmax) * 0x10001u;
-  // rint(m / s) <= zp + qmax + 1 must stay a small positive 16-bit integer for the packed steps
-  c.pad = 0;
-  c.packed = ((c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && (c.zp < 12000)) ? 1 : 0;
+  c.pad[0] = c.pad[1] = c.pad[2] = 0;
+  // Plain: no intermediate of the FMA quotient can leave the normal range, the zero-point is 0 (so no code is
+  // negative) and the largest magnitude's code needs no clamp (codes grow with the magnitude).  With a minimum
+  // of 0 the scale is fl(max / Qmax) and max / scale rounds to Qmax: no division needed to know.
+  c.plain = ((c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && c.zp == 0 &&
+             (mmin == 0.0f || __float2int_rn(__fdiv_rn(mmax, c.s)) <= c.qmax)) ? 1 : 0;
   return c;
 }
 
-// Codes of the two elements of a 16-bit pair (sign bits ignored), as two 16-bit integers.
-template <bool BF16, bool DIVIDE>
-__device__ __forceinline__ uint32_t codes2(uint32_t x, const Level& c) {
+// Codes of the two elements of a 16-bit pair (sign bits ignored), as two 16-bit integers, by the division
+// instruction: for rows that are not plain.
+template <bool BF16>
+__device__ __forceinline__ uint32_t codes2_divide(uint32_t x, const Level& c) {
   using E = Elem<BF16>;
   const float lo = fabsf(E::lo_f32(x)), hi = fabsf(E::hi_f32(x));
-  if (DIVIDE) {
-    const int klo = __vimin_s32_relu(__float2int_rn(__fdiv_rn(lo, c.s)) - c.zp, c.qmax);
-    const int khi = __vimin_s32_relu(__float2int_rn(__fdiv_rn(hi, c.s)) - c.zp, c.qmax);
-    return static_cast<uint32_t>(klo) | (static_cast<uint32_t>(khi) << 16);
-  }
-  const float q0 = __fmul_rn(lo, c.r), q1 = __fmul_rn(hi, c.r);
-  const float tlo = __fadd_rn(fmaf(fmaf(-q0, c.s, lo), c.r, q0), kRoundMagic);  // fl(lo / s), then to an integer
-  const float thi = __fadd_rn(fmaf(fmaf(-q1, c.s, hi), c.r, q1), kRoundMagic);
-  // pattern of 2^23 + k = 0x4B000000 + k, so thi * 2^16 + tlo (mod 2^32) = (0x4B00 + k_hi) << 16 | k_lo;
-  // the constant in the high half is taken off together with zp.
-  const uint32_t k2 = mad_u32(__float_as_uint(thi), 65536u, __float_as_uint(tlo));
-  return __viaddmin_s16x2_relu(k2, c.nz2, c.qm2);  // clamp(k - zp, 0, qmax) in both halves
+  const int klo = __vimin_s32_relu(__float2int_rn(__fdiv_rn(lo, c.s)) - c.zp, c.qmax);
+  const int khi = __vimin_s32_relu(__float2int_rn(__fdiv_rn(hi, c.s)) - c.zp, c.qmax);
+  return static_cast<uint32_t>(klo) | (static_cast<uint32_t>(khi) << 16);
+}
+
+// ---- plain rows: two elements at a time with the packed binary32 instructions (each lane IEEE round-to-nearest-even) ----
+__device__ __forceinline__ uint64_t pack2f(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2u(uint64_t v, uint32_t& lo, uint32_t& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+struct Level2 {
+  uint64_t r2, ns2;  // {r, r} and {-s, -s}
+};
+__device__ __forceinline__ Level2 make_level2(const Level& c) {
+  Level2 l;
+  l.r2 = pack2f(c.r, c.r);
+  l.ns2 = pack2f(-c.s, -c.s);
+  return l;
+}
+// Magnitudes of the two elements of a 16-bit pair as packed binary32.
+template <bool BF16>
+__device__ __forceinline__ uint64_t magnitudes2(uint32_t x) {
+  const uint32_t a = x & 0x7fff7fffu;
+  if (BF16) return pack2u(mad_u32(a, 65536u, 0u), a & 0xffff0000u);
+  const float2 f = __half22float2(Elem<false>::as2(a));
+  return pack2f(f.x, f.y);
+}
+// rint(fl(m / s)) + 2^23 in both lanes: q0 = fl(m r), the residual m - q0 s (one FMA, exact), q = fl(q0 + residual r),
+// then the addition that rounds to an integer.  The code is the low byte of the result's pattern.
+__device__ __forceinline__ uint64_t quotient2(uint64_t m2, const Level2& l, uint64_t magic2) {
+  const uint64_t q0 = mul2(m2, l.r2);
+  const uint64_t e = fma2(q0, l.ns2, m2);
+  const uint64_t q = fma2(e, l.r2, q0);
+  return add2(q, magic2);
+}
+// Low bytes of four patterns 2^23 + k (k < 256) as one word: bytes a.lo, b.lo, a.hi, b.hi.
+__device__ __forceinline__ uint32_t bytes4(uint64_t ta, uint64_t tb) {
+  uint32_t alo, ahi, blo, bhi;
+  unpack2u(ta, alo, ahi);
+  unpack2u(tb, blo, bhi);
+  return __byte_perm(mad_u32(blo, 256u, alo), mad_u32(bhi, 256u, ahi), 0x5410);
 }
 
 __device__ __forceinline__ uint32_t max_s16x2(uint32_t a, uint32_t b) {
@@ -151,42 +208,46 @@ __device__ __forceinline__ uint32_t split_group(uint32_t (&x)[16], uint32_t nval
   return bitmap;
 }
 
-// Pass B on one group: sum |(q0 >> sh) - q| over its 32 elements (Algorithm 1's distortion numerator).
-// The codes of two pairs are packed into four bytes, shifted and masked four at a time, and summed by the
-// byte-wise sum-of-absolute-differences instruction: 5 integer instructions per four elements.
-template <bool BF16, bool DIVIDE>
-__device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], const Level& top, const Level& low,
-                                                     int sh) {
+// Pass B on one group of a plain row: sum |(q0 >> sh) - q| over its 32 elements (Algorithm 1's distortion
+// numerator).  Four codes travel as the bytes of one word: the shift and mask take four at a time, and the
+// byte-wise sum-of-absolute-differences instruction adds the four differences.
+template <bool BF16>
+__device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], const Level2& top, const Level2& low, int sh) {
   const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+  const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
   uint32_t S = 0;
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
-    const uint32_t ct4 = __byte_perm(codes2<BF16, DIVIDE>(x[i], top), codes2<BF16, DIVIDE>(x[i + 1], top), 0x6420);
-    const uint32_t q4 = __byte_perm(codes2<BF16, DIVIDE>(x[i], low), codes2<BF16, DIVIDE>(x[i + 1], low), 0x6420);
+    const uint64_t ma = magnitudes2<BF16>(x[i]), mb = magnitudes2<BF16>(x[i + 1]);
+    const uint32_t ct4 = bytes4(quotient2(ma, top, magic2), quotient2(mb, top, magic2));
+    const uint32_t q4 = bytes4(quotient2(ma, low, magic2), quotient2(mb, low, magic2));
     S = __vsadu4((ct4 >> sh) & shmask, q4) + S;
   }
   return S;
 }
 
-// Pass B for the first lower candidate, keeping what pass C needs if that candidate fails: on return
-// tb[i] (i < 4) holds the top-level bytes (code | sign << 7) of elements 2i, 2i + 1, 8 + 2i, 8 + 2i + 1 and
-// tb[4 + i] those of the elements 16 further on.  (Any grouping of four serves the sum; this one is the
-// grouping from which two byte permutes per i give the input of the bit transpose.)
-template <bool BF16, bool DIVIDE>
-__device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], const Level& top, const Level& low, int sh,
+// Pass B for the first lower candidate, keeping what pass C needs if that candidate fails: on return tb[4h + i]
+// holds the top-level bytes (code | sign << 7) of elements 16h + 2i, 16h + 8 + 2i, 16h + 2i + 1, 16h + 8 + 2i + 1 (pair i
+// of chunks 2h and 2h + 1, low elements first) and ql the candidate's own codes in the same grouping, no signs.
+// (Any grouping of four serves the sum; this one costs the byte assembly least, and two byte permutes per i
+// turn it into the input of the bit transpose.)
+template <bool BF16>
+__device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], const Level2& top, const Level2& low, int sh,
                                                      uint32_t (&tb)[8], uint32_t (&ql)[8]) {
   const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+  const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
   uint32_t S = 0;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint32_t xa = x[8 * h + i], xb = x[8 * h + 4 + i];  // pairs i of chunks 2h and 2h + 1
-      const uint32_t ct4 = __byte_perm(codes2<BF16, DIVIDE>(xa, top), codes2<BF16, DIVIDE>(xb, top), 0x6420);
-      const uint32_t q4 = __byte_perm(codes2<BF16, DIVIDE>(xa, low), codes2<BF16, DIVIDE>(xb, low), 0x6420);
+      const uint64_t ma = magnitudes2<BF16>(xa), mb = magnitudes2<BF16>(xb);
+      const uint32_t ct4 = bytes4(quotient2(ma, top, magic2), quotient2(mb, top, magic2));
+      const uint32_t q4 = bytes4(quotient2(ma, low, magic2), quotient2(mb, low, magic2));
       S = __vsadu4((ct4 >> sh) & shmask, q4) + S;
-      tb[4 * h + i] = ct4 | (__byte_perm(xa, xb, 0x7531) & 0x80808080u);  // the sign bits sit in bytes 1 and 3 of a pair
-      ql[4 * h + i] = q4;  // the candidate's own codes, same grouping, no signs: its planes if it is the one chosen
+      tb[4 * h + i] = ct4 | (__byte_perm(xa, xb, 0x7351) & 0x80808080u);  // the sign bits sit in bytes 1 and 3 of a pair
+      ql[4 * h + i] = q4;
     }
   }
   return S;
@@ -194,17 +255,19 @@ __device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], co
 
 // Pass B for a further candidate: the top-level codes come from the bytes the first turn left.
 template <bool BF16>
-__device__ __forceinline__ uint32_t distortion_next(const uint32_t (&x)[16], const uint32_t (&tb)[8], const Level& low, int sh,
+__device__ __forceinline__ uint32_t distortion_next(const uint32_t (&x)[16], const uint32_t (&tb)[8], const Level2& low, int sh,
                                                     uint32_t (&ql)[8]) {
   // a byte of tb is code | sign << 7: shifted right by sh >= 1, the sign bit and the bits that come in from
   // the next byte all land above the mask
   const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+  const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
   uint32_t S = 0;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const uint32_t q4 = __byte_perm(codes2<BF16, false>(x[8 * h + i], low), codes2<BF16, false>(x[8 * h + 4 + i], low), 0x6420);
+      const uint32_t q4 = bytes4(quotient2(magnitudes2<BF16>(x[8 * h + i]), low, magic2),
+                                 quotient2(magnitudes2<BF16>(x[8 * h + 4 + i]), low, magic2));
       S = __vsadu4((tb[4 * h + i] >> sh) & shmask, q4) + S;
       ql[4 * h + i] = q4;
     }
@@ -217,28 +280,58 @@ __device__ __forceinline__ uint32_t distortion_next(const uint32_t (&x)[16], con
 __device__ __forceinline__ void planes_of_bytes(const uint32_t (&tb)[8], uint32_t (&r)[8]) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    r[2 * i] = __byte_perm(tb[i], tb[4 + i], 0x6420);      // byte c = element 8c + 2i
-    r[2 * i + 1] = __byte_perm(tb[i], tb[4 + i], 0x7531);  // byte c = element 8c + 2i + 1
+    r[2 * i] = __byte_perm(tb[i], tb[4 + i], 0x5410);      // byte c = element 8c + 2i
+    r[2 * i + 1] = __byte_perm(tb[i], tb[4 + i], 0x7632);  // byte c = element 8c + 2i + 1
   }
-  transpose8x32(r);
+  transpose8x32_select(r);
 }
 
-// Pass C on one group: codes at the chosen level as bytes (code | sign << 7), transposed into
+// Pass C on one group of a row whose chosen level is plain: codes as bytes (code | sign << 7), transposed into
 // bit-planes: on return r[k] = bit k of every byte, k < 7 code bits, k = 7 signs.
-template <bool BF16, bool DIVIDE>
-__device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level& lv, uint32_t (&r)[8]) {
+template <bool BF16>
+__device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level2& lv, uint32_t (&r)[8]) {
+  const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
+  uint32_t tb[8];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    // b2 of chunk j: bytes of elements 8j + 2i (byte 0) and 8j + 2i + 1 (byte 2)
-    uint32_t b2[4];
+  for (int h = 0; h < 2; ++h) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) b2[j] = codes2<BF16, DIVIDE>(x[4 * j + i], lv) | ((x[4 * j + i] >> 8) & 0x00800080u);
-    const uint32_t e = b2[1] * 256u + b2[0];  // bytes: elements 2i, 8 + 2i, 2i + 1, 8 + 2i + 1
-    const uint32_t f = b2[3] * 256u + b2[2];  // the same, 16 further on
-    r[2 * i] = __byte_perm(e, f, 0x5410);      // byte c = element 8c + 2i
-    r[2 * i + 1] = __byte_perm(e, f, 0x7632);  // byte c = element 8c + 2i + 1
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t xa = x[8 * h + i], xb = x[8 * h + 4 + i];
+      const uint32_t c4 = bytes4(quotient2(magnitudes2<BF16>(xa), lv, magic2), quotient2(magnitudes2<BF16>(xb), lv, magic2));
+      tb[4 * h + i] = c4 | (__byte_perm(xa, xb, 0x7351) & 0x80808080u);
+    }
   }
-  transpose8x32(r);
+  planes_of_bytes(tb, r);
+}
+
+// The same steps with the division instruction, for one group held in registers (the one-CTA-per-row kernel).
+template <bool BF16>
+__device__ __forceinline__ uint32_t divide_distortion_regs(const uint32_t (&x)[16], const Level& top, const Level& low, int sh) {
+  const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
+  uint32_t S = 0;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const uint32_t a = (codes2_divide<BF16>(x[i], top) >> sh) & shmask;
+    const uint32_t q = codes2_divide<BF16>(x[i], low);
+    const uint32_t d = max_s16x2(a, q) - min_s16x2(a, q);
+    S += (d & 0xffffu) + (d >> 16);
+  }
+  return S;
+}
+
+struct Planes8 {
+  uint32_t v[8];
+};
+template <bool BF16>
+__device__ __forceinline__ void divide_pack_regs(const uint32_t (&x)[16], const Level& lv, uint32_t (&r)[8]) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) r[k] = 0u;  // r[k] bit e = bit k of the byte (code | sign << 7) of element e
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const uint32_t b2 = codes2_divide<BF16>(x[i], lv) | ((x[i] >> 8) & 0x00800080u);  // elements 2i (byte 0) and 2i + 1 (byte 2)
+#pragma unroll
+    for (int k = 0; k < 8; ++k) r[k] |= (((b2 >> k) & 1u) << (2 * i)) | (((b2 >> (16 + k)) & 1u) << (2 * i + 1));
+  }
 }
 
 // The same two steps for rows that need the division instruction, written as loops over the parked
@@ -251,23 +344,20 @@ __device__ __noinline__ uint32_t rolled_distortion(const uint32_t* xw, uint32_t 
 #pragma unroll 1
   for (uint32_t i = 0; i < 16; ++i) {
     const uint32_t x = xw[4u * park_index(nt, u, i >> 2) + (i & 3u)];
-    const uint32_t a = (codes2<BF16, true>(x, top) >> sh) & shmask;
-    const uint32_t q = codes2<BF16, true>(x, low);
+    const uint32_t a = (codes2_divide<BF16>(x, top) >> sh) & shmask;
+    const uint32_t q = codes2_divide<BF16>(x, low);
     const uint32_t d = max_s16x2(a, q) - min_s16x2(a, q);
     S += (d & 0xffffu) + (d >> 16);
   }
   return S;
 }
-struct Planes8 {
-  uint32_t v[8];
-};
 template <bool BF16>
 __device__ __noinline__ Planes8 rolled_pack(const uint32_t* xw, uint32_t nt, uint32_t u, Level lv) {
   uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // r[k] bit e = bit k of the byte (code | sign << 7) of element e
 #pragma unroll 1
   for (uint32_t i = 0; i < 16; ++i) {
     const uint32_t x = xw[4u * park_index(nt, u, i >> 2) + (i & 3u)];
-    const uint32_t b2 = codes2<BF16, true>(x, lv) | ((x >> 8) & 0x00800080u);  // elements 2i (byte 0) and 2i + 1 (byte 2)
+    const uint32_t b2 = codes2_divide<BF16>(x, lv) | ((x >> 8) & 0x00800080u);  // elements 2i (byte 0) and 2i + 1 (byte 2)
 #pragma unroll
     for (int k = 0; k < 8; ++k) r[k] |= (((b2 >> k) & 1u) << (2u * i)) | (((b2 >> (16 + k)) & 1u) << (2u * i + 1u));
   }
@@ -346,7 +436,13 @@ __device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartial
     S_out[lane] = 0;
   }
   if (lane == 0) *row_cnt = total;
-  return __all_sync(kFull, lv.packed != 0) ? 0u : 1u;
+  return __all_sync(kFull, lv.plain != 0) ? 0u : 1u;
+}
+
+// The limit on device-side waits: the workspace's setting, else the built-in one.
+__device__ __forceinline__ uint32_t lookback_limit(const EncodeParams& p) {
+  const uint32_t set = *reinterpret_cast<volatile const uint32_t*>(&p.ws->poll_limit);
+  return set != 0u ? set : kLookbackPollLimit;
 }
 
 __device__ __forceinline__ unsigned long long pack_desc(uint32_t tag, uint32_t value) {
@@ -386,7 +482,7 @@ __device__ __forceinline__ uint32_t tile_state(uint32_t gen4, unsigned long long
 // 1024 than with 256).
 template <int DEPTH>
 __device__ int resolve_prefix(const EncodeParams& p, uint32_t gen4, uint32_t tile, uint32_t agg_w, uint32_t agg_o,
-                              uint32_t lane, uint32_t* excl_w, uint32_t* excl_o) {
+                              uint32_t lane, uint32_t* excl_w, uint32_t* excl_o, uint32_t poll_limit) {
   uint32_t base_w = 0, base_o = 0;  // prefix found at the end of the walk
   uint32_t part_w = 0, part_o = 0;  // this lane's share of the aggregates walked over
   if (tile > 0) {
@@ -448,7 +544,7 @@ __device__ int resolve_prefix(const EncodeParams& p, uint32_t gen4, uint32_t til
               state = tile_state(gen4, w0, w1);
             }
             if (__shfl_sync(kFull, state, 0) != 0u) break;
-            if (++polls > kLookbackPollLimit) return TSQ_ERR_TIMEOUT;
+            if (++polls > poll_limit) return TSQ_ERR_TIMEOUT;
             __nanosleep(polls < 32u ? 200u : 1000u);
           }
         }
@@ -622,9 +718,9 @@ __global__ void __launch_bounds__(1024, 1) encode_rows_kernel(const EncodeParams
 #pragma unroll
       for (int k = 0; k < UPT; ++k) {
         if (divide) {
-          S += distortion_group<BF16, true>(x[k], top, low, shn);
+          S += divide_distortion_regs<BF16>(x[k], top, low, shn);
         } else {
-          S += distortion_group<BF16, false>(x[k], top, low, shn);
+          S += distortion_group<BF16>(x[k], make_level2(top), make_level2(low), shn);
         }
       }
       S = __reduce_add_sync(kFull, S);
@@ -643,16 +739,16 @@ __global__ void __launch_bounds__(1024, 1) encode_rows_kernel(const EncodeParams
 #pragma unroll
     for (int k = 0; k < UPT; ++k) {
       if (divide) {
-        pack_group<BF16, true>(x[k], best, r[k]);
+        divide_pack_regs<BF16>(x[k], best, r[k]);
       } else {
-        pack_group<BF16, false>(x[k], best, r[k]);
+        pack_group<BF16>(x[k], make_level2(best), r[k]);
       }
     }
 
     // ---- placement: exclusive prefix sums over the tokens before this one ----
     if (warp == 0) {
       uint32_t word_off = 0, out_base = 0;
-      const int st = resolve_prefix<8>(p, gen4, tile, agg_w, row_cnt, lane, &word_off, &out_base);
+      const int st = resolve_prefix<8>(p, gen4, tile, agg_w, row_cnt, lane, &word_off, &out_base, lookback_limit(p));
       if (lane == 0) {
         sh.word_off = word_off;
         sh.out_base = out_base;
@@ -752,6 +848,9 @@ struct PipeShared {
   volatile uint32_t placed;    // rows placed
   volatile uint32_t finished;  // the compute warps are done: a_ready and packed are final
   volatile uint32_t abort;     // a wait inside the CTA ran out
+  volatile uint32_t stop[2];   // abort as thread 0 saw it before the iteration's barrier, by iteration parity: what the
+                               // compute threads act on, so that all of them leave the row loop in the same iteration
+  uint32_t wait_limit;         // polls before a handshake gives up
   uint32_t next_tile[2];       // ticket of the row after the current one, by iteration parity
 };
 
@@ -767,7 +866,7 @@ __device__ __forceinline__ bool wait_beyond(volatile uint32_t* counter, uint32_t
     if (*counter > n) return true;
     if (sh.abort != 0u) return false;
     if (may_finish && sh.finished != 0u) return *counter > n;
-    if (polls > kHandshakePollLimit) {
+    if (polls > sh.wait_limit) {
       sh.abort = 1u;
       return false;
     }
@@ -796,6 +895,11 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     sh.placed = 0u;
     sh.finished = 0u;
     sh.abort = 0u;
+    sh.stop[0] = sh.stop[1] = 0u;
+    {
+      const uint32_t lim = lookback_limit(p);
+      sh.wait_limit = lim > 0xffffffffu / kHandshakeFactor ? 0xffffffffu : lim * kHandshakeFactor;
+    }
     sh.next_tile[0] = atomicAdd(&p.ws->ticket, 1u);
   }
   __syncthreads();
@@ -814,7 +918,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     uint32_t ticket_ahead = 0xffffffffu;
     if (tid == 0 && tile_cur < p.tokens) ticket_ahead = atomicAdd(&p.ws->ticket, 1u);
 
-    for (;;) {
+    for (uint32_t it = 0u;; ++it) {
       const bool have_cur = tile_cur < p.tokens;
       if (!have_cur && !have_prev) break;
       uint32_t bitmap_cur = 0u, cnt_cur = 0u, first_cur = 0u;
@@ -864,9 +968,12 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           // pass B of row n_a - 1 needs its levels
           wait_beyond(&sh.lv_ready, n_a - 1u, sh, false, 100u);
         }
+        // The levels and placement warps may raise abort at any moment.  Thread 0 alone samples it, before the
+        // barrier, into a word that nobody else writes: every compute thread then takes the same branch.
+        sh.stop[it & 1u] = sh.abort;
       }
       compute_barrier(nt);
-      if (sh.abort != 0u) break;
+      if (sh.stop[it & 1u] != 0u) break;
       if (tid == 0) {
         __threadfence_block();
         if (have_cur) sh.a_ready = n_a + 1u;
@@ -923,7 +1030,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             }
             const int c0 = ci >= 0 ? ci : 0;
             const Level low = m.lv[c0];
-            uint32_t S = distortion_first<BF16, false>(y, top, low, bmax - p.bits[c0], tb, lb);
+            uint32_t S = distortion_first<BF16>(y, make_level2(top), make_level2(low), bmax - p.bits[c0], tb, lb);
             if (ci >= 0) {
               S = __reduce_add_sync(kFull, S);
               if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
@@ -951,7 +1058,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
                 y[4 * j + 3] = c.w;
               }
               const Level low = m.lv[ci];
-              uint32_t S = distortion_next<BF16>(y, tb, low, bmax - p.bits[ci], ql);
+              uint32_t S = distortion_next<BF16>(y, tb, make_level2(low), bmax - p.bits[ci], ql);
               S = __reduce_add_sync(kFull, S);
               if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
               compute_barrier(nt);
@@ -1053,7 +1160,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       const RowMeta& m = sh.meta[n % kMetaRing];
       const uint32_t tile = m.tile, agg_w = m.agg_w, row_cnt = m.row_cnt;
       uint32_t word_off = 0, out_base = 0;
-      const int st = resolve_prefix<1>(p, gen4, tile, agg_w, row_cnt, lane, &word_off, &out_base);
+      const int st = resolve_prefix<1>(p, gen4, tile, agg_w, row_cnt, lane, &word_off, &out_base, lookback_limit(p));
       if (st != TSQ_OK) {
         if (lane == 0) {
           publish(p, gen4 | kFlagAbort, tile, 0u, 0u);

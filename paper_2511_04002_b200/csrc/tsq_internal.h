@@ -67,7 +67,8 @@ struct WsControl {
   uint32_t enc_status;   // first encode error since init (sticky)
   uint32_t dec_status;   // first decode error since init (sticky)
   uint32_t desc_capacity;  // tiles the descriptor array holds (set by init)
-  uint32_t pad[9];
+  uint32_t poll_limit;     // polls before a device-side wait gives up; 0 = the built-in limit
+  uint32_t pad[8];
 };
 static_assert(sizeof(WsControl) == 64, "control block is 64 bytes");
 
