@@ -12,9 +12,13 @@ figure through the host-buffer entry points with the host<->device copies inside
 single-threaded CPU oracle on the same tensor; `decode_step` is the per-call latency of the
 decode-step workload (512 independent 64 x 4096 tensors).
 
-With N > 1 (one process per GPU, launched by torch.distributed.run) every rank encodes and decodes
-its own tensor: tokens are independent, there is no exchange step, so the job scales weakly with no
-collective on the data path.  `--impl reference` times the CPU oracle instead (rank 0 only).
+`workloads` carries encode / decode times of the other workloads (a few steps each, own clocks).
+
+With N > 1 every rank (one process per GPU) encodes and decodes its own tensor: tokens are independent,
+there is no exchange step, so the job scales weakly with no collective on the data path.  Started
+plainly as `python bench.py --gpus N` the script launches its N ranks itself (torch.distributed.run on
+127.0.0.1); started under torch.distributed.run it takes its rank from the environment.
+`--impl reference` times the CPU oracle instead (rank 0 only).
 """
 from __future__ import annotations
 
@@ -181,6 +185,15 @@ def cpu_baseline(x_cpu: torch.Tensor, w, budget_s: float = 12.0):
                 passes, T, H, elapsed)}
 
 
+def config_of(w, T, H, extra=None):
+    """The keys both arms print under `config` (the same for the same workload)."""
+    c = {"workload": w.name, "tokens": T, "hidden": H, "elem": w.recipe.dtype, "tau": w.tau, "bits": list(w.bits),
+         "delta": w.delta, "seed": w.seed, "tokens_per_gpu": T, "parallelism": "token ranges per GPU, no collective"}
+    if extra:
+        c.update(extra)
+    return c
+
+
 def run_reference(args, w):
     rank, world, _ = dist_env()
     if rank != 0:
@@ -205,8 +218,8 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "tokens": T, "hidden": H, "tau": w.tau, "bits": list(w.bits), "delta": w.delta,
-                   "seed": w.seed, "sample": sample_txt},
+        "config": config_of(w, T, H),
+        "sample": sample_txt,
         "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample_txt},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -284,6 +297,56 @@ def decode_step_latency(B, device, n_calls: int):
     info = plan.blob_info(bl[0])
     assert info.status == 0 and plan.workspace_status(ws) == (0, 0)
     out["payload_bytes_call0"] = info.payload_bytes
+    return out
+
+
+def time_workload(B, device, w, peak, steps=12, warmup=4, sets=None):
+    """Encode and decode times of one workload: CUDA events around every launch, buffer sets rotated so that at
+    least ~300 MB are touched between reuses of a set (inputs never found in L2), clocks sampled meanwhile."""
+    T, H = w.recipe.tokens, w.recipe.hidden
+    dt = synth.torch_dtype(w.recipe.dtype)
+    plan = B.Plan(dt, H, T, w.tau, list(w.bits), w.delta, device=device)
+    x0 = synth.make(w)
+    per_set = 2 * T * H * 2 + T * H
+    n_sets = sets or max(2, min(24, int(3e8 // per_set) + 1))
+    bufs = []
+    for k in range(n_sets):
+        x = torch.roll(x0, k, 0).cuda() if k else x0.cuda()       # the same rows in another order: same statistics
+        blob, ws = plan.alloc(T)
+        bufs.append((x, blob, ws, torch.empty_like(x)))
+    stream = torch.cuda.current_stream()
+    for i in range(warmup):
+        x, blob, ws, y = bufs[i % n_sets]
+        plan.encode(x, blob, ws); plan.decode(blob, T, y, ws)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps + 1)]
+    with ClockSampler(device, period_s=0.001) as clocks:
+        ev[0].record(stream)
+        for i in range(steps):
+            x, blob, ws, y = bufs[i % n_sets]
+            plan.encode(x, blob, ws); ev[2 * i + 1].record(stream)
+            plan.decode(blob, T, y, ws); ev[2 * i + 2].record(stream)
+        torch.cuda.synchronize()
+    enc_us = 1e3 * sum(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(steps)) / steps
+    dec_us = 1e3 * sum(ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(steps)) / steps
+    info = plan.blob_info(bufs[0][1])
+    assert info.status == 0 and plan.workspace_status(bufs[0][2]) == (0, 0), "codec reported an error on %s" % w.name
+    nbytes = T * H * 2 + info.payload_bytes
+    bits = np.bincount(bufs[0][1][64:64 + T].cpu().numpy(), minlength=9)
+    return {"tokens": T, "hidden": H, "elem": w.recipe.dtype, "bits": list(w.bits), "tau": w.tau, "steps": steps,
+            "buffer_sets": n_sets, "bytes_per_launch": nbytes, "payload_bytes": info.payload_bytes,
+            "outliers": info.total_outliers, "rows_per_bit_width": {str(b): int(bits[b]) for b in w.bits if bits[b]},
+            "encode": {"us": enc_us, "GB/s": nbytes / enc_us / 1e3, "frac": nbytes / enc_us / 1e3 / peak},
+            "decode": {"us": dec_us, "GB/s": nbytes / dec_us / 1e3, "frac": nbytes / dec_us / 1e3 / peak},
+            "clocks": clocks.summary()}
+
+
+def other_workloads(B, device, peak):
+    out = {}
+    for w in (synth.c1_prefill(), synth.c3_13b_prefill(), synth.c5_sweep_point(3, 1, 0), synth.c5_sweep_point(3, 2, 1),
+              synth.c5_sweep_point(4, 1, 0), synth.c5_sweep_point(4, 2, 1)):
+        out[w.name] = time_workload(B, device, w, peak)
+        torch.cuda.empty_cache()
     return out
 
 
@@ -408,25 +471,44 @@ def run_tsq(args, w):
         "metric": METRIC, "value": bytes_done / (total_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": args.warmup, "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "tokens": T, "hidden": H, "elem": w.recipe.dtype, "tau": w.tau,
-                   "bits": list(w.bits), "delta": w.delta, "seed": w.seed, "tokens_per_gpu": T,
-                   "parallelism": "token ranges per GPU, no collective",
-                   "l2": "rotating %d distinct input/blob/output sets (%.0f MB touched between reuses)" % (
-                       n_sets, n_sets * (2 * x_bytes + p0) / 1e6),
-                   "payload_bytes": p0, "compression_ratio": x_bytes / p0},
+        "config": config_of(w, T, H),
+        "l2": "rotating %d distinct input/blob/output sets (%.0f MB touched between reuses)" % (
+            n_sets, n_sets * (2 * x_bytes + p0) / 1e6),
+        "payload_bytes": p0, "compression_ratio": x_bytes / p0,
         "clocks": clocks.summary(), "gpu_launches": launches, "kernels": kern, "roofline": roofline,
     }
     if e2e is not None:
         line["e2e"] = e2e
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(x0, w)
-    if world == 1 and not args.no_decode_step:
+    if world == 1 and not (args.no_decode_step and args.no_workloads):
         for s in sets[1:]:
             del s.x, s.blob, s.y
+        del sets
+        torch.cuda.empty_cache()
+    if world == 1 and not args.no_decode_step:
         line["decode_step"] = decode_step_latency(B, local, args.decode_calls)
+    if world == 1 and not args.no_workloads:
+        line["workloads"] = other_workloads(B, local, peak)
     if world > 1:
         dist.destroy_process_group()
     print(json.dumps(line), flush=True)
+
+
+def launch_ranks(n: int, argv, backend_env=None) -> int:
+    """Start this script once per GPU under torch.distributed.run (rendezvous on 127.0.0.1) and return its exit code."""
+    import socket
+    import subprocess
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")                 # the communicator's set-up goes to stderr
+    if backend_env:
+        env.update(backend_env)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd, env=env)
 
 
 def main():
@@ -443,9 +525,12 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode-step", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the encode / decode times of the other workloads")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "tsq":
+        raise SystemExit(launch_ranks(args.gpus, sys.argv[1:]))
     w = workload_by_name(args.workload, args.tokens or None)
     if args.impl == "reference":
         run_reference(args, w)

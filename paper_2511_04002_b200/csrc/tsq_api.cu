@@ -345,6 +345,8 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
     // few rows (or rows too long for the pipeline): one CTA per row; a call without rows still launches
     // one CTA, which writes the header
     const int grid = tokens > 0 ? static_cast<int>(tokens) : 1;
+    // up to one CTA per SM is resident whatever the CTA's size: such a call needs no tickets
+    p.direct_tiles = tokens <= static_cast<int64_t>(plan->sms) ? 1u : 0u;
     e = launch_encode_rows(p, grid, plan->enc_threads, plan->enc_upt, static_cast<cudaStream_t>(cuda_stream));
   }
   g_launches.fetch_add(1);

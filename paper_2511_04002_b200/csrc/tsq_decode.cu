@@ -58,7 +58,7 @@ __device__ __forceinline__ void restore_units(const DecodeParams& p, const uint3
         if (static_cast<uint32_t>(k) + 1u < b) r[k] = __ldg(src + 1 + k);
       }
     }
-    transpose8x32(r);  // r[i] byte c = (code | sign << 7) of element 8c + i
+    transpose8x32_select(r);  // r[i] byte c = (code | sign << 7) of element 8c + i
     const uint32_t rot = (u >> 1) & 3u;
 #pragma unroll
     for (uint32_t j = 0; j < 4; ++j) {

@@ -643,15 +643,18 @@ struct RowShared {
   uint32_t status;     // TSQ_OK, or why the row is not written
 };
 
-template <bool BF16, int UPT>
-__global__ void __launch_bounds__(1024, 1) encode_rows_kernel(const EncodeParams p) {
+// MAXT: the largest CTA the instance is launched with (rows of up to 8192 elements get the 256-thread instance,
+// which may use four times the registers of the 1024-thread one).
+template <bool BF16, int UPT, int MAXT>
+__global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(const EncodeParams p) {
   using E = Elem<BF16>;
   __shared__ RowShared sh;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const uint32_t gen4 = (*reinterpret_cast<volatile const uint32_t*>(&p.ws->gen) + 1u) << 2;
 
   if (tid == 0) {
-    sh.tile = atomicAdd(&p.ws->ticket, 1u);
+    // a call whose rows all get a CTA at once needs no ticket: every CTA is running, so row = CTA index is safe
+    sh.tile = p.direct_tiles != 0u ? blockIdx.x : atomicAdd(&p.ws->ticket, 1u);
     sh.status = TSQ_OK;
   }
   __syncthreads();
@@ -1324,17 +1327,23 @@ cudaError_t launch_encode_pipe(const EncodeParams& p, bool full, int grid, int t
 
 cudaError_t launch_encode_rows(const EncodeParams& p, int grid, int threads, int upt, cudaStream_t stream) {
   const bool bf16 = p.dtype == TSQ_BF16;
-  if (upt == 1) {
+  if (upt == 1 && threads <= 256) {
     if (bf16) {
-      encode_rows_kernel<true, 1><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<true, 1, 256><<<grid, threads, 0, stream>>>(p);
     } else {
-      encode_rows_kernel<false, 1><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<false, 1, 256><<<grid, threads, 0, stream>>>(p);
+    }
+  } else if (upt == 1) {
+    if (bf16) {
+      encode_rows_kernel<true, 1, 1024><<<grid, threads, 0, stream>>>(p);
+    } else {
+      encode_rows_kernel<false, 1, 1024><<<grid, threads, 0, stream>>>(p);
     }
   } else {
     if (bf16) {
-      encode_rows_kernel<true, 2><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<true, 2, 1024><<<grid, threads, 0, stream>>>(p);
     } else {
-      encode_rows_kernel<false, 2><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<false, 2, 1024><<<grid, threads, 0, stream>>>(p);
     }
   }
   return cudaGetLastError();

@@ -87,6 +87,7 @@ struct EncodeParams {
   int32_t bits[8];
   int32_t s_max;                             // floor(delta * H), clamped to [-1, INT32_MAX]
   uint32_t vec_store;                        // 1: every token's plane words start on a 16-byte boundary
+  uint32_t direct_tiles;                     // one-CTA-per-row kernel: 1 = row index is the CTA index (every CTA resident)
   // pipelined kernel only: thread split, shared-memory strides (bytes; csr_cap in entries), ring depth in rows
   uint32_t compute_threads, park_stride, planes_stride, csr_cap, ring;
   uint32_t dtype;

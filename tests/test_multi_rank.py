@@ -12,6 +12,8 @@ import torch.multiprocessing as mp
 from oracle import tsq_ref as R
 from paper_2511_04002_b200 import shard, synth
 
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
 
 def test_token_ranges_partition_the_rows():
     for tokens in (0, 1, 7, 64, 8192, 8193):
@@ -63,3 +65,19 @@ def test_two_ranks_shard_without_a_data_collective(tmp_path):
 
 def test_reduce_job_without_a_process_group():
     assert shard.reduce_job(1.5, 10, 2, "cpu") == (1.5, 10.0, 2)
+
+
+def test_bench_launches_its_own_ranks(capfd):
+    """`bench.py --gpus N` started plainly launches N ranks under torch.distributed.run on 127.0.0.1.  Here, without a
+    GPU, the launcher is driven with the CPU arm: rank 0 prints the one JSON line, the other rank exits 0."""
+    import importlib.util
+    import json
+    spec = importlib.util.spec_from_file_location("bench_for_test", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    rc = bench.launch_ranks(2, ["--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "3", "--workload", "c1"])
+    assert rc == 0
+    out = capfd.readouterr().out
+    lines = [json.loads(l) for l in out.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
+    assert lines[0]["config"]["workload"].startswith("c1_") and "sample" in lines[0]
