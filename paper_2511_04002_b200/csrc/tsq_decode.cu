@@ -70,6 +70,17 @@ __device__ __forceinline__ void restore_units(const DecodeParams& p, const uint3
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const uint32_t p2 = __byte_perm(r[2 * i], r[2 * i + 1], sel);  // elements 8cc + 2i (byte 0) and 8cc + 2i + 1 (byte 2)
+        if (ZP0 && !DIRECT) {
+          // zero-point 0: the pattern of 2^23 + code is the code byte under the top byte of 2^23, two byte
+          // permutes; both products (2^23 + code) * s - 2^23 * s in one packed FMA (each lane rounds as the
+          // scalar instruction does)
+          const uint32_t c2 = p2 & 0x007f007fu;
+          const uint64_t v2 = pack2u(__byte_perm(c2, kTwo23Bits, 0x7440), __byte_perm(c2, kTwo23Bits, 0x7442));
+          float flo2, fhi2;
+          unpack2f(fma2(v2, pack2f(s, s), pack2f(neg_bias, neg_bias)), flo2, fhi2);
+          out[i] = (p2 & 0x00800080u) * 256u + E::pack_rn(flo2, fhi2);  // sign bits 7 / 23 -> 15 / 31
+          continue;
+        }
         const uint32_t clo = p2 & 0x7fu, chi = __umulhi(p2, 65536u) & 0x7fu;
         float flo, fhi;
         if (DIRECT) {

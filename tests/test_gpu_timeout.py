@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 TIMEOUT = 7
 
 
-@pytest.mark.parametrize("tokens,hidden", [(48, 512),      # one CTA per row
+@pytest.mark.parametrize("tokens,hidden", [(200, 512),     # one CTA per row, rows handed out by ticket (more rows than SMs)
                                            (700, 1024)])   # the persistent kernel for many rows
 def test_wait_runs_out_into_timeout_status_and_workspace_recovers(tokens, hidden):
     g = torch.Generator().manual_seed(tokens)
