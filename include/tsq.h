@@ -190,6 +190,32 @@ tsq_status_t tsq_decode_host(const tsq_plan_t *plan, const void *blob_host, size
                              void *y_host, void *blob_dev, void *y_dev, void *ws_dev, size_t ws_bytes,
                              void *cuda_stream);
 
+/*
+ * Size and latency models around the codec (host only, plain double arithmetic, no state).  They let a caller
+ * take the early-exit decisions of Algorithm 2 (send the KV cache or only the hidden state, compress harder)
+ * from byte counts: the model's before compression, tsq_blob_info's payload_bytes after it.  Every function
+ * returns NaN for arguments outside the stated ranges.
+ *
+ * tsq_model_kv_bits: Eq. "bkv" (Sec. II-B), bits of KV cache held on the edge when token w (>= 1) has reached
+ *   layer `layer` (1..n_layers):  2 * sum_{k<=layer} T_w Q_k + 2 * sum_{k>layer} T_{w-1} Q_k + hd * Q_layer,
+ *   with T_w = w * hd and Q_k = qa_front for k < split_layer, qa_back from the split layer on (bits per element).
+ * tsq_model_io_bits: Eq. "if_total", bits of the intermediate output: the whole of Eq. "bkv" when send_kv != 0,
+ *   else the hidden state alone, T_w * Q_layer.
+ * tsq_model_outage: P_o(R) = 1 - exp(-(2^(R/W) - 1) / gamma) (Sec. II-D.2); rate R and bandwidth W in the same
+ *   unit (bits/s and Hz), gamma the received signal-to-noise ratio (linear); all three > 0.
+ * tsq_model_latency: the epsilon-outage latency  bits / R * ceil(ln(epsilon) / ln(P_o(R)))  in seconds,
+ *   0 < epsilon < 1 (one transmission when P_o is 0, +Inf when it is 1).
+ * tsq_model_best_rate: R* = argmin over [rate_lo, rate_hi] of g(R) = ln(1 / P_o(R)) / R, by a scan of 4096
+ *   cells and golden-section refinement (the paper asks for "a simple one-dimensional search").
+ */
+double tsq_model_kv_bits(int64_t w, int32_t layer, int32_t n_layers, int32_t split_layer, int64_t hd, double qa_front,
+                         double qa_back);
+double tsq_model_io_bits(int64_t w, int32_t layer, int32_t n_layers, int32_t split_layer, int64_t hd, double qa_front,
+                         double qa_back, int32_t send_kv);
+double tsq_model_outage(double rate, double bandwidth, double snr);
+double tsq_model_latency(double bits, double rate, double bandwidth, double snr, double epsilon);
+double tsq_model_best_rate(double rate_lo, double rate_hi, double bandwidth, double snr);
+
 /* Number of kernels the library has launched in this process (all plans, all streams). */
 uint64_t tsq_kernel_launch_count(void);
 

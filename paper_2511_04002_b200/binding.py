@@ -19,7 +19,8 @@ STATUS = {0: "TSQ_OK", 1: "TSQ_ERR_INVALID_ARG", 2: "TSQ_ERR_UNSUPPORTED", 3: "T
 EXPORTS = ["tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_workspace_set_wait_limit", "tsq_encode", "tsq_encode_noalloc", "tsq_decode",
            "tsq_blob_info",
            "tsq_workspace_status", "tsq_encode_host", "tsq_decode_host", "tsq_kernel_launch_count",
-           "tsq_plan_destroy", "tsq_status_string"]
+           "tsq_plan_destroy", "tsq_status_string",
+           "tsq_model_kv_bits", "tsq_model_io_bits", "tsq_model_outage", "tsq_model_latency", "tsq_model_best_rate"]
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtsq.so")
 _lib: Optional[C.CDLL] = None
@@ -66,6 +67,14 @@ def lib() -> C.CDLL:
     for name in ("tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_workspace_set_wait_limit", "tsq_encode", "tsq_decode", "tsq_blob_info",
                  "tsq_workspace_status", "tsq_encode_host", "tsq_decode_host"):
         getattr(L, name).restype = C.c_int
+    d, i32 = C.c_double, C.c_int32
+    L.tsq_model_kv_bits.argtypes = [i64, i32, i32, i32, i64, d, d]
+    L.tsq_model_io_bits.argtypes = [i64, i32, i32, i32, i64, d, d, i32]
+    L.tsq_model_outage.argtypes = [d, d, d]
+    L.tsq_model_latency.argtypes = [d, d, d, d, d]
+    L.tsq_model_best_rate.argtypes = [d, d, d, d]
+    for name in ("tsq_model_kv_bits", "tsq_model_io_bits", "tsq_model_outage", "tsq_model_latency", "tsq_model_best_rate"):
+        getattr(L, name).restype = d
     L.tsq_kernel_launch_count.argtypes = []
     L.tsq_kernel_launch_count.restype = C.c_uint64
     L.tsq_plan_destroy.argtypes = [vp]
@@ -190,6 +199,26 @@ class Plan:
                                    blob_dev.data_ptr(), y_dev.data_ptr(), ws.data_ptr(), ws.numel(),
                                    _stream(stream))
         _check(st, "tsq_decode_host")
+
+
+def model_kv_bits(w, layer, n_layers, split_layer, hd, qa_front, qa_back) -> float:
+    return float(lib().tsq_model_kv_bits(w, layer, n_layers, split_layer, hd, qa_front, qa_back))
+
+
+def model_io_bits(w, layer, n_layers, split_layer, hd, qa_front, qa_back, send_kv) -> float:
+    return float(lib().tsq_model_io_bits(w, layer, n_layers, split_layer, hd, qa_front, qa_back, 1 if send_kv else 0))
+
+
+def model_outage(rate, bandwidth, snr) -> float:
+    return float(lib().tsq_model_outage(rate, bandwidth, snr))
+
+
+def model_latency(bits, rate, bandwidth, snr, epsilon) -> float:
+    return float(lib().tsq_model_latency(bits, rate, bandwidth, snr, epsilon))
+
+
+def model_best_rate(rate_lo, rate_hi, bandwidth, snr) -> float:
+    return float(lib().tsq_model_best_rate(rate_lo, rate_hi, bandwidth, snr))
 
 
 def kernel_launch_count() -> int:
