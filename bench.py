@@ -48,10 +48,10 @@ FALLBACK_HBM_GBS = 6650.0
 # under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
 # (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
 NCU_TRAFFIC = {
-    "encode": {"sha256": "0a591ccb46927174d99eaa8f9cda8910c211a22fb49172334b0170361d2e7c87",
-               "bytes_per_token": (134319104 + 36340480) / 8192, "hidden": 8192, "dtype": "bf16"},
-    "decode": {"sha256": "be5a19566be9449ea9a692b638af3c35bae99b39688b20c4117b9328b6eaedf3",
-               "bytes_per_token": (68642816 + 76561408) / 8192, "hidden": 8192, "dtype": "bf16"},
+    "encode": {"sha256": "001886d6afd20171571b7dfd3df8a335134ee3c39e0ab6fd5dd02181e4339736",
+               "bytes_per_token": (134290944 + 35410944) / 8192, "hidden": 8192, "dtype": "bf16"},
+    "decode": {"sha256": "d99432530c71894fb5f4258a160673f785dc4260321df5f8f055d9976ff48599",
+               "bytes_per_token": (68665600 + 76496896) / 8192, "hidden": 8192, "dtype": "bf16"},
 }
 KERNEL_NAMES = {"encode": "encode_pipe_kernel (encode_rows_kernel for few or very long rows)", "decode": "decode_kernel"}
 
