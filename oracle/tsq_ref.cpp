@@ -53,6 +53,13 @@
 //   R15 the reconstruction is the binary32 product rounded once (RNE) to the
 //       16-bit input type.
 //
+// Variant "signed values" (flag 1, an alternative reading of Sec. II-C.2): Eq. "Proposed" is applied to the
+// signed inliers themselves, without Algorithm 1 lines 1-2 (no sign / magnitude split): the per-token min and
+// max are those of the signed values of T_below (outlier slots count as +0), a b-bit level spends all b bits on
+// the code, Q_max(b) = 2^b - 1, the zero-point rint(T_min / s) may be negative, and there is no sign plane
+// (plane k = bit k of the code).  Everything else (TS, descent, distortion test, placement, restore
+// (code + zp) * s rounded once to the 16-bit type) is as above.  The blob header marks it in bits[7].
+//
 // Parity pins: see tests/test_oracle_*.py.  The paper prints no numeric example
 // for TS, AIQ or TAB-Q, so the choice among readings R1-R6 is pinned only by the
 // internal consistency of its equations ("parity unpinned" for that choice);
@@ -164,6 +171,14 @@ uint16_t float_to_bf16_rne_nonneg(float f) {
   return (uint16_t)hi;
 }
 
+uint16_t float_to_raw16_nonneg(int dtype, float f);
+// signed binary32 -> 16-bit pattern, round to nearest even on the magnitude, sign kept
+uint16_t float_to_raw16_signed(int dtype, float f) {
+  const uint32_t u = float_to_bits(f);
+  const uint16_t mag = float_to_raw16_nonneg(dtype, bits_to_float(u & 0x7fffffffu));
+  return (uint16_t)(mag | ((u >> 31) << 15));
+}
+
 float raw16_to_float(int dtype, uint16_t r) {
   return dtype == kF16 ? f16_to_float(r) : bf16_to_float(r);
 }
@@ -269,6 +284,33 @@ void aiq(const float* m, int64_t H, float mmin, float mmax, int b, float* s_out,
   *zp_out = zp;
 }
 
+// ---- variant "signed values": AIQ on the signed inliers, Q_max = 2^b - 1 ---------------------------------
+// v[j] = the signed value of T_below (outlier slots +0).
+void signed_values(int dtype, const uint16_t* row, int64_t H, const uint8_t* is_out, float* v) {
+  for (int64_t j = 0; j < H; ++j) v[j] = is_out[j] ? 0.0f : raw16_to_float(dtype, row[j]);
+}
+
+void aiq_signed(const float* v, int64_t H, float vmin, float vmax, int b, float* s_out, int32_t* zp_out, int32_t* q) {
+  const int32_t qmax = (1 << b) - 1;
+  const float range = vmax - vmin;
+  float s;
+  if (range > 0.0f) {
+    s = range / (float)qmax;
+  } else {
+    const float c = std::fabs(vmax);  // a constant row: one level at the value itself (R10 carried over)
+    s = (c > 0.0f) ? c : 1.0f;
+  }
+  const int32_t zp = (int32_t)std::rint(vmin / s);
+  for (int64_t j = 0; j < H; ++j) {
+    int32_t c = (int32_t)std::rint(v[j] / s) - zp;
+    if (c < 0) c = 0;
+    if (c > qmax) c = qmax;
+    q[j] = c;
+  }
+  *s_out = s;
+  *zp_out = zp;
+}
+
 void row_min_max(const float* m, int64_t H, float* mmin, float* mmax) {
   float lo = m[0], hi = m[0];
   for (int64_t j = 1; j < H; ++j) {
@@ -300,19 +342,26 @@ struct RowResult {
 };
 
 RowResult tabq_row(const float* m, int64_t H, const int32_t* bits, int n_bits, int64_t s_max,
-                   std::vector<int32_t>& q0, std::vector<int32_t>& q, std::vector<int32_t>& qbest) {
+                   std::vector<int32_t>& q0, std::vector<int32_t>& q, std::vector<int32_t>& qbest, bool signed_values_variant = false) {
   float mmin, mmax;
   row_min_max(m, H, &mmin, &mmax);
   const int bmax = bits[n_bits - 1];
   RowResult best;
   best.b = bmax;
-  aiq(m, H, mmin, mmax, bmax, &best.s, &best.zp, q0.data());
+  const auto quantise = [&](int b, float* s, int32_t* zp, int32_t* out) {
+    if (signed_values_variant) {
+      aiq_signed(m, H, mmin, mmax, b, s, zp, out);
+    } else {
+      aiq(m, H, mmin, mmax, b, s, zp, out);
+    }
+  };
+  quantise(bmax, &best.s, &best.zp, q0.data());
   qbest = q0;
   for (int i = n_bits - 2; i >= 0; --i) {
     const int b = bits[i];
     float s;
     int32_t zp;
-    aiq(m, H, mmin, mmax, b, &s, &zp, q.data());
+    quantise(b, &s, &zp, q.data());
     const int64_t S = distortion_sum(q0.data(), q.data(), H, bmax, b);
     if (S > s_max) break;  // delta > Delta: stop, keep the last passing level
     best.b = b;
@@ -347,10 +396,12 @@ int tsq_ref_layout(int hidden, long long tokens, int bmax, long long max_outlier
 
 // Encode x[tokens][hidden] (raw 16-bit patterns, host memory) into blob (host memory).
 // The whole blob is zero-filled first, so unused capacity reads as zero.
-int tsq_ref_encode(int dtype, int hidden, long long tokens, float tau, const int32_t* bits,
-                   int n_bits, float delta, long long max_outliers, const uint16_t* x,
-                   uint8_t* blob, unsigned long long blob_bytes) {
+int tsq_ref_encode_ex(int dtype, int hidden, long long tokens, float tau, const int32_t* bits,
+                      int n_bits, float delta, long long max_outliers, int flags, const uint16_t* x,
+                      uint8_t* blob, unsigned long long blob_bytes) {
   if ((dtype != kF16 && dtype != kBF16) || !check_bits(bits, n_bits) || !blob) return kInvalidArg;
+  if (flags != 0 && flags != 1) return kInvalidArg;
+  const bool sv = flags == 1;  // variant "signed values"
   if (tau != tau || delta != delta) return kInvalidArg;
   if (tokens > 0 && !x) return kInvalidArg;
   const int bmax = bits[n_bits - 1];
@@ -389,7 +440,8 @@ int tsq_ref_encode(int dtype, int hidden, long long tokens, float tau, const int
       }
       ++out_ptr;
     }
-    const RowResult r = tabq_row(m.data(), H, bits, n_bits, s_max, q0, q, qbest);
+    if (sv) signed_values(dtype, row, H, is_out.data(), m.data());  // m now holds the signed values of T_below
+    const RowResult r = tabq_row(m.data(), H, bits, n_bits, s_max, q0, q, qbest, sv);
     o_bits[t] = (uint8_t)r.b;
     o_scale[t] = r.s;
     o_zp[t] = r.zp;
@@ -400,6 +452,12 @@ int tsq_ref_encode(int dtype, int hidden, long long tokens, float tau, const int
     for (int64_t j = 0; j < H; ++j) {
       const uint64_t g = (uint64_t)j >> 5;
       const uint32_t bit = 1u << (j & 31);
+      if (sv) {  // no sign plane: plane k = bit k of the b-bit code
+        for (int k = 0; k < r.b; ++k) {
+          if ((qbest[j] >> k) & 1) wrow[g * r.b + k] |= bit;
+        }
+        continue;
+      }
       if (sg[j]) wrow[g * r.b] |= bit;
       for (int k = 0; k < r.b - 1; ++k) {
         if ((qbest[j] >> k) & 1) wrow[g * r.b + 1 + k] |= bit;
@@ -419,6 +477,7 @@ int tsq_ref_encode(int dtype, int hidden, long long tokens, float tau, const int
   h.tokens = (uint32_t)tokens;
   h.n_bits = (uint32_t)n_bits;
   for (int i = 0; i < n_bits; ++i) h.bits[i] = (uint8_t)bits[i];
+  h.bits[7] = (uint8_t)flags;  // n_bits <= 7: the last entry is free and carries the variant
   h.tau = tau;
   h.delta = delta;
   h.total_words = word_off;
@@ -426,6 +485,21 @@ int tsq_ref_encode(int dtype, int hidden, long long tokens, float tau, const int
   h.status = status;
   h.outlier_capacity = (uint32_t)L.outlier_capacity;
   std::memcpy(blob, &h, sizeof h);
+  return kOk;
+}
+
+int tsq_ref_encode(int dtype, int hidden, long long tokens, float tau, const int32_t* bits,
+                   int n_bits, float delta, long long max_outliers, const uint16_t* x,
+                   uint8_t* blob, unsigned long long blob_bytes) {
+  return tsq_ref_encode_ex(dtype, hidden, tokens, tau, bits, n_bits, delta, max_outliers, 0, x, blob, blob_bytes);
+}
+
+// Variant "signed values": AIQ at level b on a row of binary32 signed values (already threshold-split).
+int tsq_ref_aiq_signed(const float* v, int hidden, int b, float* s, int32_t* zp, int32_t* q) {
+  if (!v || hidden < 1 || b < 2 || b > 8 || !s || !zp || !q) return kInvalidArg;
+  float vmin, vmax;
+  row_min_max(v, hidden, &vmin, &vmax);
+  aiq_signed(v, hidden, vmin, vmax, b, s, zp, q);
   return kOk;
 }
 
@@ -438,6 +512,8 @@ int tsq_ref_decode(const uint8_t* blob, unsigned long long blob_bytes, uint16_t*
   if (h.dtype != (uint32_t)kF16 && h.dtype != (uint32_t)kBF16) return kCorruptBlob;
   if (h.n_bits < 1 || h.n_bits > 7) return kCorruptBlob;
   if (h.status != kOk) return (int)h.status;
+  if (h.bits[7] > 1) return kCorruptBlob;
+  const bool sv = h.bits[7] == 1;
   const int bmax = h.bits[h.n_bits - 1];
   Layout L;
   if (!make_layout(h.hidden, h.tokens, bmax, h.outlier_capacity, &L)) return kCorruptBlob;
@@ -471,6 +547,12 @@ int tsq_ref_decode(const uint8_t* blob, unsigned long long blob_bytes, uint16_t*
     for (int64_t j = 0; j < H; ++j) {
       const uint64_t g = (uint64_t)j >> 5;
       const int sh = (int)(j & 31);
+      if (sv) {
+        int32_t q = 0;
+        for (int k = 0; k < b; ++k) q |= (int32_t)((wrow[g * b + k] >> sh) & 1u) << k;
+        yrow[j] = float_to_raw16_signed(dtype, (float)(q + zp) * s);  // signed product, rounded once
+        continue;
+      }
       int32_t q = 0;
       for (int k = 0; k < b - 1; ++k) q |= (int32_t)((wrow[g * b + 1 + k] >> sh) & 1u) << k;
       const uint32_t sign = (wrow[g * b] >> sh) & 1u;

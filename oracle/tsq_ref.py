@@ -35,6 +35,11 @@ def lib() -> C.CDLL:
         L.tsq_ref_encode.argtypes = [C.c_int, C.c_int, C.c_longlong, C.c_float, i32p, C.c_int, C.c_float,
                                      C.c_longlong, u16p, u8p, C.c_ulonglong]
         L.tsq_ref_encode.restype = C.c_int
+        L.tsq_ref_encode_ex.argtypes = [C.c_int, C.c_int, C.c_longlong, C.c_float, i32p, C.c_int, C.c_float,
+                                        C.c_longlong, C.c_int, u16p, u8p, C.c_ulonglong]
+        L.tsq_ref_encode_ex.restype = C.c_int
+        L.tsq_ref_aiq_signed.argtypes = [f32p, C.c_int, C.c_int, f32p, i32p, i32p]
+        L.tsq_ref_aiq_signed.restype = C.c_int
         L.tsq_ref_decode.argtypes = [u8p, C.c_ulonglong, u16p]
         L.tsq_ref_decode.restype = C.c_int
         L.tsq_ref_ts_row.argtypes = [C.c_int, u16p, C.c_int, C.c_float, f32p, u8p, u8p, C.POINTER(C.c_longlong)]
@@ -76,8 +81,9 @@ def layout(hidden: int, tokens: int, bmax: int, max_outliers: int = 0) -> Dict[s
 
 
 def encode(x_raw: np.ndarray, dtype: int, tau: float, bits: Sequence[int], delta: float = 0.2,
-           max_outliers: int = 0) -> np.ndarray:
-    """x_raw: uint16 [tokens, hidden]. Returns the blob as a uint8 array."""
+           max_outliers: int = 0, signed_values: bool = False) -> np.ndarray:
+    """x_raw: uint16 [tokens, hidden]. Returns the blob as a uint8 array. signed_values: the variant that
+    quantises the signed inliers (no sign plane, Q_max = 2^b - 1)."""
     x_raw = np.ascontiguousarray(x_raw, dtype=np.uint16)
     assert x_raw.ndim == 2
     tokens, hidden = x_raw.shape
@@ -85,8 +91,8 @@ def encode(x_raw: np.ndarray, dtype: int, tau: float, bits: Sequence[int], delta
     bmax = int(b[-1]) if b.size and 2 <= int(b[-1]) <= 8 else 8   # invalid lists are rejected by the C side
     lay = layout(hidden, tokens, bmax, max_outliers)
     blob = np.empty(lay["total"], dtype=np.uint8)
-    st = lib().tsq_ref_encode(dtype, hidden, tokens, tau, _ptr(b, C.c_int32), len(b), delta, max_outliers,
-                              _ptr(x_raw, C.c_uint16), _ptr(blob, C.c_uint8), blob.size)
+    st = lib().tsq_ref_encode_ex(dtype, hidden, tokens, tau, _ptr(b, C.c_int32), len(b), delta, max_outliers,
+                                 1 if signed_values else 0, _ptr(x_raw, C.c_uint16), _ptr(blob, C.c_uint8), blob.size)
     if st:
         raise OracleError(st)
     return blob
@@ -108,7 +114,7 @@ def header(blob: np.ndarray) -> Dict[str, object]:
     u32 = h.view(np.uint32)
     return {
         "magic": int(u32[0]), "version": int(u32[1]), "dtype": int(u32[2]), "hidden": int(u32[3]),
-        "tokens": int(u32[4]), "n_bits": int(u32[5]), "bits": [int(v) for v in h[24:32]],
+        "tokens": int(u32[4]), "n_bits": int(u32[5]), "bits": [int(v) for v in h[24:31]] + [0], "variant": int(h[31]),
         "tau": float(h[32:36].view(np.float32)[0]), "delta": float(h[36:40].view(np.float32)[0]),
         "total_words": int(h[40:48].view(np.uint64)[0]), "total_outliers": int(h[48:56].view(np.uint64)[0]),
         "status": int(u32[14]), "outlier_capacity": int(u32[15]),
@@ -154,6 +160,17 @@ def aiq(m: np.ndarray, b: int):
     s = C.c_float(0)
     zp = C.c_int32(0)
     st = lib().tsq_ref_aiq(_ptr(m, C.c_float), m.size, b, C.byref(s), C.byref(zp), _ptr(q, C.c_int32))
+    if st:
+        raise OracleError(st)
+    return float(s.value), int(zp.value), q
+
+
+def aiq_signed(v: np.ndarray, b: int):
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    q = np.empty(v.size, np.int32)
+    s = C.c_float(0)
+    zp = C.c_int32(0)
+    st = lib().tsq_ref_aiq_signed(_ptr(v, C.c_float), v.size, b, C.byref(s), C.byref(zp), _ptr(q, C.c_int32))
     if st:
         raise OracleError(st)
     return float(s.value), int(zp.value), q
