@@ -300,12 +300,12 @@ def decode_step_latency(B, device, n_calls: int):
     return out
 
 
-def time_workload(B, device, w, peak, steps=12, warmup=4, sets=None):
+def time_workload(B, device, w, peak, steps=12, warmup=4, sets=None, variant=0):
     """Encode and decode times of one workload: CUDA events around every launch, buffer sets rotated so that at
     least ~300 MB are touched between reuses of a set (inputs never found in L2), clocks sampled meanwhile."""
     T, H = w.recipe.tokens, w.recipe.hidden
     dt = synth.torch_dtype(w.recipe.dtype)
-    plan = B.Plan(dt, H, T, w.tau, list(w.bits), w.delta, device=device)
+    plan = B.Plan(dt, H, T, w.tau, list(w.bits), w.delta, device=device, variant=variant)
     x0 = synth.make(w)
     per_set = 2 * T * H * 2 + T * H
     n_sets = sets or max(2, min(24, int(3e8 // per_set) + 1))
@@ -334,6 +334,7 @@ def time_workload(B, device, w, peak, steps=12, warmup=4, sets=None):
     nbytes = T * H * 2 + info.payload_bytes
     bits = np.bincount(bufs[0][1][64:64 + T].cpu().numpy(), minlength=9)
     return {"tokens": T, "hidden": H, "elem": w.recipe.dtype, "bits": list(w.bits), "tau": w.tau, "steps": steps,
+            "variant": "signed_values" if variant else "magnitudes",
             "buffer_sets": n_sets, "bytes_per_launch": nbytes, "payload_bytes": info.payload_bytes,
             "outliers": info.total_outliers, "rows_per_bit_width": {str(b): int(bits[b]) for b in w.bits if bits[b]},
             "encode": {"us": enc_us, "GB/s": nbytes / enc_us / 1e3, "frac": nbytes / enc_us / 1e3 / peak},
@@ -347,6 +348,10 @@ def other_workloads(B, device, peak):
               synth.c5_sweep_point(4, 1, 0), synth.c5_sweep_point(4, 2, 1)):
         out[w.name] = time_workload(B, device, w, peak)
         torch.cuda.empty_cache()
+    # the signed-values variant of the codec (AIQ on the signed inliers, no sign plane) on the c3 tensor
+    w = synth.c3_13b_prefill()
+    out[w.name + "_signed_values"] = time_workload(B, device, w, peak, variant=B.VARIANT_SIGNED_VALUES)
+    torch.cuda.empty_cache()
     return out
 
 

@@ -47,6 +47,19 @@ typedef enum {
 
 typedef enum { TSQ_F16 = 0, TSQ_BF16 = 1 } tsq_dtype_t;
 
+/*
+ * Which values Eq. "Proposed" quantises.
+ *   TSQ_VARIANT_MAGNITUDES     Algorithm 1 as printed: sign and magnitude are separated first, a b-bit level is
+ *                              one sign bit + a (b-1)-bit code of the magnitude, Q_max = 2^(b-1) - 1.
+ *   TSQ_VARIANT_SIGNED_VALUES  Eq. "Proposed" applied to the signed inliers themselves (the other reading of
+ *                              Sec. II-C.2, without Algorithm 1's first two steps): min and max are those of
+ *                              the signed values of T_below (outlier slots count as +0), a b-bit level is a
+ *                              b-bit code, Q_max = 2^b - 1, the zero-point may be negative, no sign plane.
+ * A blob records its variant (header byte bits[7]) and is decoded only by a plan of the same variant.
+ */
+#define TSQ_VARIANT_MAGNITUDES 0
+#define TSQ_VARIANT_SIGNED_VALUES 1
+
 typedef struct {
   size_t blob_bytes;      /* bytes of the blob buffer for `tokens` rows (capacity, not payload) */
   size_t workspace_bytes; /* bytes of the workspace the plan needs (independent of `tokens`) */
@@ -66,17 +79,23 @@ typedef struct {
  * of the last two sections are meaningful).  WPP = ceil(hidden / 32).
  *
  *   header   64 B  u32 magic 'TSQ1' | u32 version=1 | u32 dtype | u32 hidden | u32 tokens |
- *                  u32 n_bits | u8 bits[8] | f32 tau | f32 delta | u64 total_words |
+ *                  u32 n_bits | u8 bits[7] | u8 variant | f32 tau | f32 delta | u64 total_words |
  *                  u64 total_outliers | u32 status | u32 outlier_capacity
- *   bits     u8  [tokens]      chosen bit-width b* (1 sign bit + (b*-1)-bit magnitude code)
+ *   bits     u8  [tokens]      chosen bit-width b* (1 sign bit + (b*-1)-bit magnitude code; signed-values
+ *                              variant: a b*-bit code)
  *   scale    f32 [tokens]      AIQ scale s
- *   zp       i32 [tokens]      AIQ zero-point, restore = (code + zp) * s
+ *   zp       i32 [tokens]      AIQ zero-point, restore = (code + zp) * s.  The decoder accepts 0 <= zp < 2^22
+ *                              (|zp| < 2^22 in the signed-values variant) and reports any other value as
+ *                              TSQ_ERR_CORRUPT_BLOB: 16-bit inputs cannot produce more (the minimum over
+ *                              the scale is at most 2^11 Q_max, below 2^19), and the bound keeps code + zp
+ *                              exact in binary32
  *   word_off u32 [tokens+1]    exclusive prefix sum of b* x WPP
  *   out_ptr  u32 [tokens+1]    CSR row pointers (exclusive prefix sum of per-token outlier counts)
  *   words    u32 [tokens x bmax x WPP]  token t owns b* x WPP words from word_off[t], interleaved
  *                  per group of 32 elements: word g*b* + k is plane k of elements 32g .. 32g+31,
  *                  plane 0 = sign bits of the inliers, plane 1+k = bit k of the magnitude codes;
- *                  bit i of a group's word belongs to element 32g + i; pad bits are 0
+ *                  bit i of a group's word belongs to element 32g + i; pad bits are 0.  Signed-values
+ *                  variant: plane k = bit k of the code, no sign plane
  *   outl     u32 [outlier_capacity]     (column << 16) | original 16-bit pattern, columns ascending
  */
 
@@ -98,6 +117,15 @@ typedef struct {
  */
 tsq_status_t tsq_plan(tsq_plan_t **out, int device, tsq_dtype_t dtype, int32_t hidden, int64_t max_tokens,
                       float tau, const int32_t *bits, int32_t n_bits, float delta, int64_t max_outliers);
+
+/*
+ * The same with the variant chosen (TSQ_VARIANT_*; tsq_plan is this call with TSQ_VARIANT_MAGNITUDES).  Any other
+ * value is TSQ_ERR_INVALID_ARG.  Every other call takes plans of either variant.  The signed-values variant is
+ * served by the one-CTA-per-row encoder at every size and by the division instruction (no fast steps).
+ */
+tsq_status_t tsq_plan_variant(tsq_plan_t **out, int device, tsq_dtype_t dtype, int32_t hidden, int64_t max_tokens,
+                              float tau, const int32_t *bits, int32_t n_bits, float delta, int64_t max_outliers,
+                              int32_t variant);
 
 /* Buffer sizes for a call with `tokens` rows (0 <= tokens <= max_tokens). `out` is HOST. */
 tsq_status_t tsq_plan_sizes(const tsq_plan_t *plan, int64_t tokens, tsq_sizes_t *out);

@@ -57,7 +57,8 @@
 // signed inliers themselves, without Algorithm 1 lines 1-2 (no sign / magnitude split): the per-token min and
 // max are those of the signed values of T_below (outlier slots count as +0), a b-bit level spends all b bits on
 // the code, Q_max(b) = 2^b - 1, the zero-point rint(T_min / s) may be negative, and there is no sign plane
-// (plane k = bit k of the code).  Everything else (TS, descent, distortion test, placement, restore
+// (plane k = bit k of the code); a range T_max - T_min that overflows binary32 counts as the largest finite
+// binary32.  Everything else (TS, descent, distortion test, placement, restore
 // (code + zp) * s rounded once to the 16-bit type) is as above.  The blob header marks it in bits[7].
 //
 // Parity pins: see tests/test_oracle_*.py.  The paper prints no numeric example
@@ -292,7 +293,10 @@ void signed_values(int dtype, const uint16_t* row, int64_t H, const uint8_t* is_
 
 void aiq_signed(const float* v, int64_t H, float vmin, float vmax, int b, float* s_out, int32_t* zp_out, int32_t* q) {
   const int32_t qmax = (1 << b) - 1;
-  const float range = vmax - vmin;
+  float range = vmax - vmin;
+  // Two finite values of opposite sign can lie further apart than binary32 holds (bf16 rows spanning more than
+  // 3.4e38): the difference then counts as the largest finite binary32, so that scale and codes stay finite.
+  if (range > 3.40282346638528859811704183484516925e+38f) range = 3.40282346638528859811704183484516925e+38f;
   float s;
   if (range > 0.0f) {
     s = range / (float)qmax;

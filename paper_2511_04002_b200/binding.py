@@ -16,7 +16,9 @@ F16, BF16 = 0, 1
 STATUS = {0: "TSQ_OK", 1: "TSQ_ERR_INVALID_ARG", 2: "TSQ_ERR_UNSUPPORTED", 3: "TSQ_ERR_BUFFER_TOO_SMALL",
           4: "TSQ_ERR_CUDA", 5: "TSQ_ERR_CORRUPT_BLOB", 6: "TSQ_ERR_OUTLIER_OVERFLOW", 7: "TSQ_ERR_TIMEOUT"}
 
-EXPORTS = ["tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_workspace_set_wait_limit", "tsq_encode", "tsq_encode_noalloc", "tsq_decode",
+VARIANT_MAGNITUDES, VARIANT_SIGNED_VALUES = 0, 1
+
+EXPORTS = ["tsq_plan", "tsq_plan_variant", "tsq_plan_sizes", "tsq_workspace_init", "tsq_workspace_set_wait_limit", "tsq_encode", "tsq_encode_noalloc", "tsq_decode",
            "tsq_blob_info",
            "tsq_workspace_status", "tsq_encode_host", "tsq_decode_host", "tsq_kernel_launch_count",
            "tsq_plan_destroy", "tsq_status_string",
@@ -53,6 +55,7 @@ def lib() -> C.CDLL:
     vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
     L.tsq_plan.argtypes = [C.POINTER(vp), C.c_int, C.c_int, C.c_int32, i64, C.c_float, C.POINTER(C.c_int32),
                            C.c_int32, C.c_float, i64]
+    L.tsq_plan_variant.argtypes = L.tsq_plan.argtypes + [C.c_int32]
     L.tsq_plan_sizes.argtypes = [vp, i64, C.POINTER(_Sizes)]
     L.tsq_workspace_init.argtypes = [vp, vp, sz, vp]
     L.tsq_workspace_set_wait_limit.argtypes = [vp, C.c_uint32, vp]
@@ -64,7 +67,7 @@ def lib() -> C.CDLL:
     L.tsq_workspace_status.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), vp]
     L.tsq_encode_host.argtypes = [vp, vp, i64, vp, sz, C.POINTER(C.c_uint64), vp, vp, vp, sz, vp]
     L.tsq_decode_host.argtypes = [vp, vp, sz, i64, vp, vp, vp, vp, sz, vp]
-    for name in ("tsq_plan", "tsq_plan_sizes", "tsq_workspace_init", "tsq_workspace_set_wait_limit", "tsq_encode", "tsq_decode", "tsq_blob_info",
+    for name in ("tsq_plan", "tsq_plan_variant", "tsq_plan_sizes", "tsq_workspace_init", "tsq_workspace_set_wait_limit", "tsq_encode", "tsq_decode", "tsq_blob_info",
                  "tsq_workspace_status", "tsq_encode_host", "tsq_decode_host"):
         getattr(L, name).restype = C.c_int
     d, i32 = C.c_double, C.c_int32
@@ -119,12 +122,17 @@ class Plan:
     """tsq_plan_t wrapper. Methods are the C calls of the same name with pointers filled in."""
 
     def __init__(self, dtype: torch.dtype, hidden: int, max_tokens: int, tau: float, bits: Sequence[int],
-                 delta: float = 0.2, max_outliers: int = 0, device: int = 0):
+                 delta: float = 0.2, max_outliers: int = 0, device: int = 0, variant: int = VARIANT_MAGNITUDES):
         self._h = C.c_void_p()
         arr = (C.c_int32 * len(bits))(*bits)
-        st = lib().tsq_plan(C.byref(self._h), device, dtype_code(dtype), hidden, max_tokens, tau, arr, len(bits),
-                            delta, max_outliers)
+        if variant == VARIANT_MAGNITUDES:
+            st = lib().tsq_plan(C.byref(self._h), device, dtype_code(dtype), hidden, max_tokens, tau, arr, len(bits),
+                                delta, max_outliers)
+        else:
+            st = lib().tsq_plan_variant(C.byref(self._h), device, dtype_code(dtype), hidden, max_tokens, tau, arr,
+                                        len(bits), delta, max_outliers, variant)
         _check(st, "tsq_plan")
+        self.variant = variant
         self.dtype, self.hidden, self.max_tokens, self.device = dtype, hidden, max_tokens, device
         self.tau, self.bits, self.delta, self.max_outliers = tau, tuple(bits), delta, max_outliers
 

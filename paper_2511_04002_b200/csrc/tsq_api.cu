@@ -95,6 +95,7 @@ struct tsq_plan {
   int32_t bmax;
   int32_t s_max;
   uint32_t thr16;
+  uint32_t variant;                 // 0: sign + magnitude codes; 1: codes of the signed values
   int threads;                      // decoder CTA size, one group per thread
   int threads_half, dec_blocks_half; // the same with two groups per thread, and its resident CTAs per SM
   int enc_threads, enc_upt;         // row-at-a-time encoder: CTA size and 32-element groups per thread
@@ -130,8 +131,14 @@ uint64_t tsq_kernel_launch_count(void) { return g_launches.load(); }
 
 tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t hidden, int64_t max_tokens, float tau,
                       const int32_t* bits, int32_t n_bits, float delta, int64_t max_outliers) {
+  return tsq_plan_variant(out, device, dtype, hidden, max_tokens, tau, bits, n_bits, delta, max_outliers, TSQ_VARIANT_MAGNITUDES);
+}
+
+tsq_status_t tsq_plan_variant(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t hidden, int64_t max_tokens, float tau,
+                              const int32_t* bits, int32_t n_bits, float delta, int64_t max_outliers, int32_t variant) {
   if (!out) return TSQ_ERR_INVALID_ARG;
   *out = nullptr;
+  if (variant != TSQ_VARIANT_MAGNITUDES && variant != TSQ_VARIANT_SIGNED_VALUES) return TSQ_ERR_INVALID_ARG;
   if (dtype != TSQ_F16 && dtype != TSQ_BF16) return TSQ_ERR_INVALID_ARG;
   if (!bits || n_bits < 1 || n_bits > kMaxCand) return TSQ_ERR_INVALID_ARG;
   for (int i = 0; i < n_bits; ++i) {
@@ -161,6 +168,7 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
   p->n_bits = n_bits;
   for (int i = 0; i < 8; ++i) p->bits[i] = i < n_bits ? bits[i] : 0;
   p->bmax = bmax;
+  p->variant = static_cast<uint32_t>(variant);
   const double smax = std::floor(static_cast<double>(delta) * static_cast<double>(hidden));
   p->s_max = smax < -1.0 ? -1 : (smax > 2147483647.0 ? 2147483647 : static_cast<int32_t>(smax));
   p->thr16 = threshold_pattern(dtype, tau);
@@ -214,7 +222,9 @@ tsq_status_t tsq_plan(tsq_plan_t** out, int device, tsq_dtype_t dtype, int32_t h
     p->pipe_smem = 0;
     int base_blocks = 0;
     uint32_t base_ring = 0;
-    for (uint32_t per_group = 2u; ok && per_group <= 4u && p->pipe_threads <= kPipeMaxThreads; per_group += 2u) {
+    // (the signed-values variant has no pipelined kernel: its calls all take the one-CTA-per-row kernel)
+    for (uint32_t per_group = 2u; ok && variant == TSQ_VARIANT_MAGNITUDES && per_group <= 4u && p->pipe_threads <= kPipeMaxThreads;
+         per_group += 2u) {
       const uint32_t cap = per_group * p->pipe_compute;
       const auto smem_for = [&](uint32_t ring) {
         return 3u * static_cast<size_t>(p->pipe_park) + ring * (static_cast<size_t>(p->pipe_planes) + 4u * static_cast<size_t>(cap));
@@ -327,6 +337,7 @@ tsq_status_t tsq_encode(const tsq_plan_t* plan, const void* x_dev, int64_t token
   p.s_max = plan->s_max;
   p.vec_store = (plan->units % 4u == 0u) ? 1u : 0u;
   p.dtype = static_cast<uint32_t>(plan->dtype);
+  p.variant = plan->variant;
   p.tau = plan->tau;
   p.delta = plan->delta;
 
@@ -375,6 +386,7 @@ tsq_status_t tsq_decode(const tsq_plan_t* plan, const void* blob_dev, size_t blo
   p.chunks = plan->chunks;
   p.bmax = static_cast<uint32_t>(plan->bmax);
   p.dtype = static_cast<uint32_t>(plan->dtype);
+  p.variant = plan->variant;
   p.blob_bytes = blob_bytes;
   const bool many_rows = tokens >= 3 * static_cast<int64_t>(plan->sms) * plan->dec_blocks_half;
   const cudaError_t e = launch_decode(p, static_cast<int>(tokens), many_rows ? plan->threads_half : plan->threads,

@@ -100,6 +100,39 @@ __device__ __forceinline__ void restore_units(const DecodeParams& p, const uint3
   }
 }
 
+// The same for a blob of the signed-values variant: plane k = bit k of the code (no sign plane), the value is
+// (code + zp) * s with a zero-point of either sign: conversion and one multiplication, rounded once to 16 bits.
+template <bool BF16>
+__device__ __noinline__ void restore_units_signed_values(const DecodeParams& p, const uint32_t* words, uint32_t b, float s,
+                                                         int32_t zp) {
+  using E = Elem<BF16>;
+  extern __shared__ __align__(128) unsigned char smem_dyn[];
+  uint4* stage4 = reinterpret_cast<uint4*>(smem_dyn);
+  for (uint32_t u = threadIdx.x; u < p.units; u += blockDim.x) {
+    uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const uint32_t* src = words + static_cast<size_t>(u) * b;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (static_cast<uint32_t>(k) < b) r[k] = __ldg(src + k);
+    }
+    transpose8x32_select(r);  // r[i] byte c = code of element 8c + i
+#pragma unroll
+    for (uint32_t cc = 0; cc < 4; ++cc) {
+      const uint32_t cidx = 4u * u + cc;
+      if (cidx >= p.chunks) continue;
+      const uint32_t sel = cc * 0x1111u + 0x4400u;
+      uint32_t out[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t p2 = __byte_perm(r[2 * i], r[2 * i + 1], sel);  // elements 8cc + 2i (bytes 0, 1) and 8cc + 2i + 1 (bytes 2, 3)
+        const int clo = static_cast<int>(p2 & 0xffu), chi = static_cast<int>(p2 >> 24);
+        out[i] = E::pack_rn(__fmul_rn(__int2float_rn(clo + zp), s), __fmul_rn(__int2float_rn(chi + zp), s));
+      }
+      stage4[cidx] = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+  }
+}
+
 template <bool BF16>
 __global__ void __launch_bounds__(kMaxThreads) decode_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char smem_dyn[];  // one output row
@@ -118,6 +151,7 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(const DecodeParams 
   }
   const bool header_ok = h->dtype == p.dtype && h->hidden == p.hidden && h->tokens == p.tokens && h->n_bits >= 1u &&
                          h->n_bits <= static_cast<uint32_t>(kMaxCand) && h->bits[(h->n_bits - 1u) & 7u] == p.bmax &&
+                         h->bits[7] == p.variant &&
                          h->outlier_capacity == static_cast<uint32_t>(p.lay.outlier_capacity) &&
                          h->total_words <= p.lay.words_capacity && h->total_outliers <= p.lay.outlier_capacity;
   if (!header_ok) {
@@ -135,7 +169,8 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(const DecodeParams 
   const uint32_t p1 = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_out_ptr)[t + 1];
   const unsigned long long span = static_cast<unsigned long long>(b) * p.lay.wpp;
   const bool row_ok = b >= 2u && b <= p.bmax && wo + span <= h->total_words && wo_next == wo + span && p0 <= p1 &&
-                      p1 <= h->total_outliers && (p1 - p0) <= p.hidden && zp >= 0 && zp < (1 << 22);
+                      p1 <= h->total_outliers && (p1 - p0) <= p.hidden && zp < (1 << 22) &&
+                      zp >= (p.variant != 0u ? 1 - (1 << 22) : 0);
   if (!row_ok) {
     if (tid == 0) record_decode_error(p, TSQ_ERR_CORRUPT_BLOB);
     return;
@@ -143,7 +178,9 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(const DecodeParams 
 
   const uint32_t* words = reinterpret_cast<const uint32_t*>(p.blob + p.lay.off_words) + wo;
   // 2^23 * s must stay finite for the conversion-free path; huge scales take the plain one.
-  if (s > 0x1p100f) {
+  if (p.variant != 0u) {
+    restore_units_signed_values<BF16>(p, words, b, s, zp);
+  } else if (s > 0x1p100f) {
     restore_units<BF16, true, false>(p, words, b, s, zp);
   } else if (zp == 0) {
     restore_units<BF16, false, true>(p, words, b, s, zp);

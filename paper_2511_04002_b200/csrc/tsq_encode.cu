@@ -93,12 +93,34 @@ __device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
   return c;
 }
 
-// Codes of the two elements of a 16-bit pair (sign bits ignored), as two 16-bit integers, by the division
-// instruction: for rows that are not plain.
-template <bool BF16>
+// The signed-values variant (Eq. "Proposed" on the signed inliers): Q_max = 2^b - 1, the zero-point may be
+// negative, a constant row takes its own magnitude as the scale.  Never plain: the division instruction does it.
+__device__ __forceinline__ Level make_level_signed(float vmin, float vmax, int b) {
+  Level c;
+  c.qmax = (1 << b) - 1;
+  // two finite values of opposite sign can lie further apart than binary32 holds: the largest finite value then
+  const float range = fminf(__fsub_rn(vmax, vmin), 3.40282346638528859811704183484516925e+38f);
+  const float a = fabsf(vmax);
+  c.s = range > 0.0f ? __fdiv_rn(range, static_cast<float>(c.qmax)) : (a > 0.0f ? a : 1.0f);
+  c.zp = __float2int_rn(__fdiv_rn(vmin, c.s));
+  c.r = 0.0f;
+  c.plain = 0;
+  c.pad[0] = c.pad[1] = c.pad[2] = 0;
+  return c;
+}
+
+// 16-bit patterns of signed values <-> 16-bit keys that order like the values (-0 just below +0).
+__device__ __forceinline__ uint32_t order_keys2(uint32_t v2) {
+  return v2 ^ 0x80008000u ^ (((v2 >> 15) & 0x10001u) * 0x7fffu);
+}
+__device__ __forceinline__ uint32_t pattern_of_key(uint32_t key) { return (key & 0x8000u) ? key ^ 0x8000u : key ^ 0xffffu; }
+
+// Codes of the two elements of a 16-bit pair, as two 16-bit integers, by the division instruction: for rows
+// that are not plain.  SV = false: codes of the magnitudes (sign bits ignored); SV = true: of the signed values.
+template <bool BF16, bool SV = false>
 __device__ __forceinline__ uint32_t codes2_divide(uint32_t x, const Level& c) {
   using E = Elem<BF16>;
-  const float lo = fabsf(E::lo_f32(x)), hi = fabsf(E::hi_f32(x));
+  const float lo = SV ? E::lo_f32(x) : fabsf(E::lo_f32(x)), hi = SV ? E::hi_f32(x) : fabsf(E::hi_f32(x));
   const int klo = __vimin_s32_relu(__float2int_rn(__fdiv_rn(lo, c.s)) - c.zp, c.qmax);
   const int khi = __vimin_s32_relu(__float2int_rn(__fdiv_rn(hi, c.s)) - c.zp, c.qmax);
   return static_cast<uint32_t>(klo) | (static_cast<uint32_t>(khi) << 16);
@@ -277,14 +299,18 @@ __device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level2
 }
 
 // The same steps with the division instruction, for one group held in registers (the one-CTA-per-row kernel).
-template <bool BF16>
-__device__ __forceinline__ uint32_t divide_distortion_regs(const uint32_t (&x)[16], const Level& top, const Level& low, int sh) {
+// (SV: the zeros past the end of a row would get non-zero codes under a negative zero-point, so only the
+// first `pairs` registers, the ones inside the row, count.)
+template <bool BF16, bool SV = false>
+__device__ __forceinline__ uint32_t divide_distortion_regs(const uint32_t (&x)[16], const Level& top, const Level& low, int sh,
+                                                           uint32_t pairs = 16u) {
   const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
   uint32_t S = 0;
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    const uint32_t a = (codes2_divide<BF16>(x[i], top) >> sh) & shmask;
-    const uint32_t q = codes2_divide<BF16>(x[i], low);
+    if (SV && static_cast<uint32_t>(i) >= pairs) continue;
+    const uint32_t a = (codes2_divide<BF16, SV>(x[i], top) >> sh) & shmask;
+    const uint32_t q = codes2_divide<BF16, SV>(x[i], low);
     const uint32_t d = max_s16x2(a, q) - min_s16x2(a, q);
     S += (d & 0xffffu) + (d >> 16);
   }
@@ -294,13 +320,14 @@ __device__ __forceinline__ uint32_t divide_distortion_regs(const uint32_t (&x)[1
 struct Planes8 {
   uint32_t v[8];
 };
-template <bool BF16>
+template <bool BF16, bool SV = false>
 __device__ __forceinline__ void divide_pack_regs(const uint32_t (&x)[16], const Level& lv, uint32_t (&r)[8]) {
 #pragma unroll
-  for (int k = 0; k < 8; ++k) r[k] = 0u;  // r[k] bit e = bit k of the byte (code | sign << 7) of element e
+  for (int k = 0; k < 8; ++k) r[k] = 0u;  // r[k] bit e = bit k of the byte (code | sign << 7; SV: the 8-bit code) of element e
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    const uint32_t b2 = codes2_divide<BF16>(x[i], lv) | ((x[i] >> 8) & 0x00800080u);  // elements 2i (byte 0) and 2i + 1 (byte 2)
+    // elements 2i (byte 0) and 2i + 1 (byte 2)
+    const uint32_t b2 = codes2_divide<BF16, SV>(x[i], lv) | (SV ? 0u : ((x[i] >> 8) & 0x00800080u));
 #pragma unroll
     for (int k = 0; k < 8; ++k) r[k] |= (((b2 >> k) & 1u) << (2 * i)) | (((b2 >> (16 + k)) & 1u) << (2 * i + 1));
   }
@@ -365,7 +392,23 @@ __device__ __forceinline__ void fetch_group(const EncodeParams& p, uint4* xpark,
 }
 
 // The b* plane words of one group, in blob order (plane 0 = sign, plane 1 + k = code bit k), to dst.
+// SV: plane k = code bit k, no sign plane.
+template <bool SV = false>
 __device__ __forceinline__ void store_planes(uint32_t* dst, const uint32_t (&r)[8], int bstar, bool vec) {
+  if (SV) {
+    if (vec && bstar == 8) {
+      reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[0], r[1], r[2], r[3]);
+      reinterpret_cast<uint4*>(dst)[1] = make_uint4(r[4], r[5], r[6], r[7]);
+    } else if (vec && bstar == 4) {
+      reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[0], r[1], r[2], r[3]);
+    } else {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        if (q < bstar) dst[q] = r[q];
+      }
+    }
+    return;
+  }
   if (vec && bstar == 8) {
     reinterpret_cast<uint4*>(dst)[0] = make_uint4(r[7], r[0], r[1], r[2]);
     reinterpret_cast<uint4*>(dst)[1] = make_uint4(r[3], r[4], r[5], r[6]);
@@ -387,7 +430,7 @@ template <int NW>  // the most warps that contribute
 struct RowPartials {
   uint32_t warp_min[NW], warp_max[NW], warp_cnt[NW];  // warp_cnt becomes an exclusive scan
 };
-template <bool BF16, int NW>
+template <bool BF16, int NW, bool SV = false>
 __device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartials<NW>& part, uint32_t nwarps, uint32_t lane,
                                                Level* lv_out, int* S_out, uint32_t* row_cnt) {
   using E = Elem<BF16>;
@@ -402,7 +445,10 @@ __device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartial
   }
   if (lane < nwarps) part.warp_cnt[lane] = incl - wc;
   const uint32_t total = __shfl_sync(kFull, incl, 31);
-  const Level lv = make_level(E::pattern_f32(pmin), E::pattern_f32(pmax), p.bits[min(lane, static_cast<uint32_t>(p.n_bits - 1))]);
+  // SV: the partial results are order keys of signed values
+  const int b = p.bits[min(lane, static_cast<uint32_t>(p.n_bits - 1))];
+  const Level lv = SV ? make_level_signed(E::pattern_f32(pattern_of_key(pmin)), E::pattern_f32(pattern_of_key(pmax)), b)
+                      : make_level(E::pattern_f32(pmin), E::pattern_f32(pmax), b);
   if (lane < static_cast<uint32_t>(p.n_bits)) {
     lv_out[lane] = lv;
     S_out[lane] = 0;
@@ -540,7 +586,8 @@ __device__ void write_header(const EncodeParams& p, unsigned long long total_wor
   h->tokens = p.tokens;
   h->n_bits = static_cast<uint32_t>(p.n_bits);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) h->bits[i] = (i < p.n_bits) ? static_cast<uint8_t>(p.bits[i]) : 0;
+  for (int i = 0; i < 7; ++i) h->bits[i] = (i < p.n_bits) ? static_cast<uint8_t>(p.bits[i]) : 0;
+  h->bits[7] = static_cast<uint8_t>(p.variant);  // at most seven candidates: the last entry carries the variant
   h->tau = p.tau;
   h->delta = p.delta;
   h->total_words = total_words;
@@ -616,8 +663,9 @@ struct RowShared {
 };
 
 // MAXT: the largest CTA the instance is launched with (rows of up to 8192 elements get the 256-thread instance,
-// which may use four times the registers of the 1024-thread one).
-template <bool BF16, int UPT, int MAXT>
+// which may use four times the registers of the 1024-thread one).  SV: the signed-values variant, which this
+// kernel alone serves, with the division instruction throughout.
+template <bool BF16, int UPT, int MAXT, bool SV>
 __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(const EncodeParams p) {
   using E = Elem<BF16>;
   __shared__ RowShared sh;
@@ -661,6 +709,22 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(
       bitmap[k] = split_group<BF16>(x[k], nvalid[k], thr2, mn2, mx2);
       cnt += __popc(bitmap[k]);
     }
+    if (SV) {
+      // min / max of the signed values of T_below instead (outlier slots are +0 by now): as order keys
+      mn2 = 0xffffffffu;
+      mx2 = 0u;
+#pragma unroll
+      for (int k = 0; k < UPT; ++k) {
+#pragma unroll
+        for (uint32_t i = 0; i < 16; ++i) {
+          if ((i >> 2) < nvalid[k]) {
+            const uint32_t key2 = order_keys2(x[k][i]);
+            mn2 = __vminu2(mn2, key2);
+            mx2 = __vmaxu2(mx2, key2);
+          }
+        }
+      }
+    }
     {
       const uint32_t mnv = __reduce_min_sync(kFull, min(mn2 & 0xffffu, mn2 >> 16));
       const uint32_t mxv = __reduce_max_sync(kFull, max(mx2 & 0xffffu, mx2 >> 16));
@@ -676,11 +740,11 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(
     // ---- AIQ parameters of every candidate level (lane i of warp 0 takes candidate i) ----
     const int bmax = p.bits[p.n_bits - 1];
     if (warp == 0) {
-      const uint32_t divide = row_levels<BF16>(p, sh.part, nwarps, lane, sh.lv, sh.S, &sh.row_cnt);
+      const uint32_t divide = row_levels<BF16, 32, SV>(p, sh.part, nwarps, lane, sh.lv, sh.S, &sh.row_cnt);
       if (lane == 0) sh.divide = divide;
     }
     __syncthreads();
-    const bool divide = sh.divide != 0u;
+    const bool divide = SV || sh.divide != 0u;
 
     // ---- Algorithm 1: descend the candidate list while the distortion stays within tolerance ----
     const Level top = sh.lv[p.n_bits - 1];
@@ -692,7 +756,9 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(
       uint32_t S = 0;
 #pragma unroll
       for (int k = 0; k < UPT; ++k) {
-        if (divide) {
+        if (SV) {
+          S += divide_distortion_regs<BF16, true>(x[k], top, low, shn, 4u * nvalid[k]);
+        } else if (divide) {
           S += divide_distortion_regs<BF16>(x[k], top, low, shn);
         } else {
           S += distortion_group<BF16>(x[k], make_level2(top), make_level2(low), shn);
@@ -713,7 +779,14 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(
     uint32_t r[UPT][8];
 #pragma unroll
     for (int k = 0; k < UPT; ++k) {
-      if (divide) {
+      if (SV) {
+        divide_pack_regs<BF16, true>(x[k], best, r[k]);
+        if (nvalid[k] < 4u) {  // pad bits stay 0: the zeros past the end of the row got the code of the value 0
+          const uint32_t inside = (1u << (8u * nvalid[k])) - 1u;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) r[k][q] &= inside;
+        }
+      } else if (divide) {
         divide_pack_regs<BF16>(x[k], best, r[k]);
       } else {
         pack_group<BF16>(x[k], make_level2(best), r[k]);
@@ -743,7 +816,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(
 #pragma unroll
       for (int k = 0; k < UPT; ++k) {
         const uint32_t u = UPT * tid + k;
-        if (u < p.units) store_planes(wrow + static_cast<size_t>(u) * bstar, r[k], bstar, p.vec_store != 0u);
+        if (u < p.units) store_planes<SV>(wrow + static_cast<size_t>(u) * bstar, r[k], bstar, p.vec_store != 0u);
       }
       if (tid == 0) write_token_fields(p, tile, bstar, best.s, best.zp, word_off + agg_w, out_base + row_cnt);
       // ---- CSR entries of T_above: ascending columns, original patterns (read again from the input) ----
@@ -1297,26 +1370,35 @@ cudaError_t launch_encode_pipe(const EncodeParams& p, bool full, int grid, int t
   return cudaGetLastError();
 }
 
-cudaError_t launch_encode_rows(const EncodeParams& p, int grid, int threads, int upt, cudaStream_t stream) {
+template <bool SV>
+static void launch_rows_variant(const EncodeParams& p, int grid, int threads, int upt, cudaStream_t stream) {
   const bool bf16 = p.dtype == TSQ_BF16;
   if (upt == 1 && threads <= 256) {
     if (bf16) {
-      encode_rows_kernel<true, 1, 256><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<true, 1, 256, SV><<<grid, threads, 0, stream>>>(p);
     } else {
-      encode_rows_kernel<false, 1, 256><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<false, 1, 256, SV><<<grid, threads, 0, stream>>>(p);
     }
   } else if (upt == 1) {
     if (bf16) {
-      encode_rows_kernel<true, 1, 1024><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<true, 1, 1024, SV><<<grid, threads, 0, stream>>>(p);
     } else {
-      encode_rows_kernel<false, 1, 1024><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<false, 1, 1024, SV><<<grid, threads, 0, stream>>>(p);
     }
   } else {
     if (bf16) {
-      encode_rows_kernel<true, 2, 1024><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<true, 2, 1024, SV><<<grid, threads, 0, stream>>>(p);
     } else {
-      encode_rows_kernel<false, 2, 1024><<<grid, threads, 0, stream>>>(p);
+      encode_rows_kernel<false, 2, 1024, SV><<<grid, threads, 0, stream>>>(p);
     }
+  }
+}
+
+cudaError_t launch_encode_rows(const EncodeParams& p, int grid, int threads, int upt, cudaStream_t stream) {
+  if (p.variant != 0u) {
+    launch_rows_variant<true>(p, grid, threads, upt, stream);
+  } else {
+    launch_rows_variant<false>(p, grid, threads, upt, stream);
   }
   return cudaGetLastError();
 }

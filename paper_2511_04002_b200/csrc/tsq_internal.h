@@ -91,6 +91,7 @@ struct EncodeParams {
   // pipelined kernel only: thread split, shared-memory strides (bytes; csr_cap in entries), ring depth in rows
   uint32_t compute_threads, park_stride, planes_stride, csr_cap, ring;
   uint32_t dtype;
+  uint32_t variant;                          // 0: sign + magnitude codes; 1: codes of the signed values (one-CTA-per-row kernel only)
   float tau, delta;
 };
 
@@ -101,6 +102,7 @@ struct DecodeParams {
   BlobLayout lay;
   uint32_t tokens, hidden, units, chunks;
   uint32_t bmax, dtype;
+  uint32_t variant;
   unsigned long long blob_bytes;
 };
 

@@ -46,13 +46,13 @@ def assert_blobs_equal(gpu_blob: np.ndarray, ref_blob: np.ndarray) -> None:
 
 
 def full_parity(x_cpu: torch.Tensor, tau: float, bits, delta: float = 0.2, max_outliers: int = 0,
-                plan: B.Plan = None, check_cross: bool = True):
+                plan: B.Plan = None, check_cross: bool = True, variant: int = 0):
     """Encode and decode on both sides; every byte must agree. Returns (gpu blob, reference blob)."""
     T, H = x_cpu.shape
     raw = synth.raw_u16(x_cpu)
-    ref_blob = R.encode(raw, dt_code(x_cpu), tau, list(bits), delta, max_outliers)
+    ref_blob = R.encode(raw, dt_code(x_cpu), tau, list(bits), delta, max_outliers, signed_values=variant == 1)
     if plan is None:
-        plan = B.Plan(x_cpu.dtype, H, max(T, 1), tau, list(bits), delta, max_outliers)
+        plan = B.Plan(x_cpu.dtype, H, max(T, 1), tau, list(bits), delta, max_outliers, variant=variant)
     blob_dev, gpu_blob, ws = gpu_encode(plan, x_cpu)
     assert gpu_blob.size == ref_blob.size
     assert_blobs_equal(gpu_blob, ref_blob)

@@ -41,6 +41,8 @@ def test_plan_argument_errors_need_no_gpu():
     bad = (ctypes.c_int32 * 2)(4, 4)
     assert L.tsq_plan(None, 0, 0, 256, 4, 6.0, bits, 3, 0.2, 0) == 1
     assert L.tsq_plan(ctypes.byref(h), 0, 5, 256, 4, 6.0, bits, 3, 0.2, 0) == 1            # dtype
+    assert L.tsq_plan_variant(ctypes.byref(h), 0, 0, 256, 4, 6.0, bits, 3, 0.2, 0, 2) == 1  # variant
+    assert L.tsq_plan_variant(ctypes.byref(h), 0, 0, 256, 4, 6.0, bits, 3, 0.2, 0, -1) == 1
     assert L.tsq_plan(ctypes.byref(h), 0, 0, 256, 4, 6.0, bad, 2, 0.2, 0) == 1             # not increasing
     assert L.tsq_plan(ctypes.byref(h), 0, 0, 100, 4, 6.0, bits, 3, 0.2, 0) == 2            # hidden % 8
     assert L.tsq_plan(ctypes.byref(h), 0, 0, 256, 4, float("nan"), bits, 3, 0.2, 0) == 1   # tau

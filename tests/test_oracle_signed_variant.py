@@ -72,6 +72,17 @@ def test_constant_rows():
     assert np.array_equal(R.decode(R.encode(raw, R.F16, INF, [3, 8], signed_values=True)), raw)
 
 
+def test_range_beyond_binary32_counts_as_the_largest_finite_value():
+    v = raw_to_f32(f32_to_raw(np.array([-3.0e38, 3.0e38, 0.0], np.float32), R.BF16), R.BF16)
+    fmax = np.finfo(np.float32).max
+    s, zp, q = R.aiq_signed(v, 2)
+    assert np.float32(s) == np.float32(fmax) / np.float32(3)
+    assert zp == int(np.rint(np.float32(v[0]) / np.float32(s))) == -3
+    assert q.tolist() == [0, 3, 3]                               # rint(2.6) + 3 = 6 is clamped; 0 + 3 = 3
+    y = R.decode(R.encode(f32_to_raw(v, R.BF16).reshape(1, 3), R.BF16, INF, [2], signed_values=True))
+    assert np.all(~np.isnan(raw_to_f32(y[0], R.BF16)))
+
+
 # ---------------------------------------------------------------- reduction to the magnitude variant
 
 @pytest.mark.parametrize("b", [2, 3, 4, 7])
