@@ -391,6 +391,23 @@ __device__ __forceinline__ void fetch_group(const EncodeParams& p, uint4* xpark,
   cp_async_commit();
 }
 
+// The CSR entries (column << 16 | original pattern) of the elements of one group that `bm` flags, in
+// ascending column order, from the group's 64 bytes as they stand in the input (v[j] = chunk j): f(entry) is
+// called once per flagged element.  All 32 positions are visited under a predicate: no data-dependent loads.
+template <typename F>
+__device__ __forceinline__ void for_each_flagged(uint32_t bm, const uint4 (&v)[4], uint32_t col0, F&& f) {
+#pragma unroll
+  for (uint32_t j = 0; j < 4; ++j) {
+    const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+    for (uint32_t i = 0; i < 4; ++i) {
+      const uint32_t e = 8u * j + 2u * i;
+      if ((bm >> e) & 1u) f(((col0 + e) << 16) | (w[i] & 0xffffu));
+      if ((bm >> (e + 1u)) & 1u) f(((col0 + e + 1u) << 16) | (w[i] >> 16));
+    }
+  }
+}
+
 // The b* plane words of one group, in blob order (plane 0 = sign, plane 1 + k = code bit k), to dst.
 // SV: plane k = code bit k, no sign plane.
 template <bool SV = false>
@@ -886,6 +903,7 @@ struct RowMeta {
   uint32_t bstar, agg_w;
   float scale;
   int zp;
+  uint32_t heavy;  // 0, or 1 + the side buffer that holds the row's outlier bitmaps (more outliers than a list holds)
 };
 
 struct PipeShared {
@@ -900,6 +918,15 @@ struct PipeShared {
                                // compute threads act on, so that all of them leave the row loop in the same iteration
   uint32_t wait_limit;         // polls before a handshake gives up
   uint32_t next_tile[2];       // ticket of the row after the current one, by iteration parity
+  // Rows with more outliers than a ring slot's list holds: the compute threads leave the groups' bitmaps in one of two
+  // side buffers, the placement warp posts the row's CSR offset there once it is resolved, and the compute threads
+  // write the entries themselves, all at once, at the top of a later iteration.
+  uint32_t heavy_bm[2][kPipeMaxThreads - 64];
+  uint32_t heavy_wcnt[2][(kPipeMaxThreads - 64) / 32];  // exclusive scan of the warps' outlier counts
+  uint32_t heavy_tile[2];
+  volatile uint32_t heavy_base[2];   // out_ptr[tile], from the placement warp
+  volatile uint32_t heavy_posted;    // such rows whose offset has been posted
+  volatile uint32_t heavy_seen[2];   // heavy_posted as thread 0 saw it before the iteration's barrier, by iteration parity
 };
 
 __device__ __forceinline__ void compute_barrier(uint32_t nthreads) {
@@ -944,6 +971,8 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     sh.finished = 0u;
     sh.abort = 0u;
     sh.stop[0] = sh.stop[1] = 0u;
+    sh.heavy_posted = 0u;
+    sh.heavy_seen[0] = sh.heavy_seen[1] = 0u;
     {
       const uint32_t lim = lookback_limit(p);
       sh.wait_limit = lim > 0xffffffffu / kHandshakeFactor ? 0xffffffffu : lim * kHandshakeFactor;
@@ -960,6 +989,40 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     uint32_t n_a = 0u;       // rows of this CTA that finished pass A; n_a - have_prev of them are packed
     uint32_t bitmap_prev = 0u, cnt_prev = 0u, first_prev = 0u;  // outliers of the thread's group in row n_a - 1
     uint32_t slot = 0u;      // ring slot of the next row to be packed: (rows packed so far) mod p.ring
+    uint32_t heavy_filled = 0u, heavy_done = 0u;  // rows put into / written out of the side buffers (the same in every thread)
+    // The CSR entries of the row in side buffer k, to their place in the blob: every thread takes its own group.
+    const auto emit_heavy = [&](uint32_t k) {
+      const uint32_t bm = sh.heavy_bm[k][u];
+      const uint32_t wbase = sh.heavy_wcnt[k][warp];
+      const uint32_t tile_h = sh.heavy_tile[k];
+      const uint32_t base = sh.heavy_base[k];
+      const uint32_t cnt = __popc(bm);
+      uint32_t incl = cnt;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(kFull, incl, d);
+        if (lane >= static_cast<uint32_t>(d)) incl += v;
+      }
+      if (bm != 0u) {
+        unsigned long long at = static_cast<unsigned long long>(base) + wbase + (incl - cnt);
+        const uint4* g = reinterpret_cast<const uint4*>(p.x + static_cast<size_t>(tile_h) * p.hidden) + 4u * u;
+        const uint32_t nv = FULL ? 4u : group_chunks(p, u);
+        uint4 v[4];
+#pragma unroll
+        for (uint32_t j = 0; j < 4; ++j) v[j] = j < nv ? g[j] : make_uint4(0u, 0u, 0u, 0u);
+        uint32_t* o_outl = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_outl);
+        bool overflow = false;
+        for_each_flagged(bm, v, 32u * u, [&](uint32_t entry) {
+          if (at < p.lay.outlier_capacity) {
+            o_outl[at] = entry;
+          } else {
+            overflow = true;
+          }
+          ++at;
+        });
+        if (overflow) atomicCAS(&p.ws->err, 0u, static_cast<uint32_t>(TSQ_ERR_OUTLIER_OVERFLOW));
+      }
+    };
     if (tile_cur < p.tokens) fetch_group(p, xpark, tile_cur, 0u, u, FULL ? 4u : group_chunks(p, u));
     // thread 0: the ticket of the row after tile_cur, asked for a whole iteration before it is needed
     // (the round trip of the atomic is longer than pass A)
@@ -1019,9 +1082,15 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         // The levels and placement warps may raise abort at any moment.  Thread 0 alone samples it, before the
         // barrier, into a word that nobody else writes: every compute thread then takes the same branch.
         sh.stop[it & 1u] = sh.abort;
+        sh.heavy_seen[it & 1u] = sh.heavy_posted;
       }
       compute_barrier(nt);
       if (sh.stop[it & 1u] != 0u) break;
+      const uint32_t heavy_done_before = heavy_done;  // a side buffer emptied in this iteration is refilled in a later one
+      if (heavy_done < heavy_filled && sh.heavy_seen[it & 1u] > heavy_done) {
+        emit_heavy(heavy_done & 1u);
+        ++heavy_done;
+      }
       if (tid == 0) {
         __threadfence_block();
         if (have_cur) sh.a_ready = n_a + 1u;
@@ -1124,9 +1193,12 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         }
         const uint32_t row_cnt = m.row_cnt;
         const uint32_t agg_w = static_cast<uint32_t>(bstar) * p.lay.wpp;
+        // more outliers than the slot's list holds: into a side buffer when one is free
+        const bool to_heavy = row_cnt > p.csr_cap && heavy_filled - heavy_done_before < 2u;
         if (tid == 0) {
           // the row's sizes are known: let the rows behind it see them
           publish_aggregate(p, gen4, tile_prev, agg_w, row_cnt);
+          m.heavy = to_heavy ? 1u + (heavy_filled & 1u) : 0u;
           m.bstar = static_cast<uint32_t>(bstar);
           m.agg_w = agg_w;
           m.scale = m.lv[best_ci].s;
@@ -1139,6 +1211,18 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         const bool slot_free = n < p.ring || wait_beyond(&sh.placed, n - p.ring, sh, false, 100u);
         // ---- planes of the chosen level into the row's slot, in blob order ----
         if (slot_free && (FULL || u < p.units)) store_planes(planes + slot * (p.planes_stride / 4u) + u * static_cast<uint32_t>(bstar), r, bstar, true);
+        // ---- a row with more outliers than the list holds leaves its groups' bitmaps in a side buffer, or, when
+        //      both are taken, in the list itself (it has room for at least two words per compute thread), where
+        //      the placement warp makes the entries from them ----
+        if (to_heavy) {
+          const uint32_t k = heavy_filled & 1u;
+          sh.heavy_bm[k][u] = bitmap_prev;
+          if (lane == 0) sh.heavy_wcnt[k][warp] = m.part.warp_cnt[warp];
+          if (tid == 0) sh.heavy_tile[k] = tile_prev;
+          ++heavy_filled;
+        } else if (slot_free && row_cnt > p.csr_cap) {
+          csr[slot * p.csr_cap + u] = bitmap_prev;
+        }
         // ---- CSR entries of T_above into the row's list: ascending columns, original patterns ----
         const uint32_t flagged = __ballot_sync(kFull, cnt_prev != 0u);
         if (flagged != 0u) {
@@ -1161,10 +1245,20 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             uint32_t bm = bitmap_prev;
             list[at++] = ((32u * u + static_cast<uint32_t>(__ffs(bm) - 1)) << 16) | first_prev;
             bm &= bm - 1u;
-            while (bm != 0u) {  // further outliers of the group: read from the input again
-              const uint32_t e = 32u * u + static_cast<uint32_t>(__ffs(bm) - 1);
-              bm &= bm - 1u;
-              list[at++] = (e << 16) | x16[e];
+            if (__popc(bm) <= 2) {
+              while (bm != 0u) {  // further outliers of the group: read from the input again
+                const uint32_t e = 32u * u + static_cast<uint32_t>(__ffs(bm) - 1);
+                bm &= bm - 1u;
+                list[at++] = (e << 16) | x16[e];
+              }
+            } else {
+              // many: the group's 64 bytes in one round trip instead of one dependent load per outlier
+              const uint4* g = reinterpret_cast<const uint4*>(x16) + 4u * u;
+              const uint32_t nv = FULL ? 4u : group_chunks(p, u);
+              uint4 v[4];
+#pragma unroll
+              for (uint32_t j = 0; j < 4; ++j) v[j] = j < nv ? g[j] : make_uint4(0u, 0u, 0u, 0u);
+              for_each_flagged(bm, v, 32u * u, [&](uint32_t entry) { list[at++] = entry; });
             }
           }
         }
@@ -1184,6 +1278,16 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       sh.packed = n_a - (have_prev ? 1u : 0u);  // have_prev is still set only when the loop was left by an abort
       __threadfence_block();
       sh.finished = 1u;
+    }
+    // rows still in the side buffers: wait for the placement warp to post their offsets
+    while (heavy_done < heavy_filled) {
+      if (tid == 0) sh.heavy_seen[0] = wait_beyond(&sh.heavy_posted, heavy_done, sh, false, 200u) ? 1u : 0u;
+      compute_barrier(nt);
+      const bool posted = sh.heavy_seen[0] != 0u;
+      if (posted) emit_heavy(heavy_done & 1u);
+      ++heavy_done;
+      compute_barrier(nt);  // before thread 0 writes heavy_seen[0] again
+      if (!posted) break;   // the CTA aborted
     }
   } else if (warp == nwarps) {
     // ================================ levels warp ================================
@@ -1236,7 +1340,14 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         if (row_cnt != 0u) {
           uint32_t* o_outl = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_outl);
           bool overflow = false;
-          if (row_cnt <= p.csr_cap) {
+          if (m.heavy != 0u) {
+            // the compute threads write this row's entries: tell them where
+            if (lane == 0) {
+              sh.heavy_base[m.heavy - 1u] = out_base;
+              __threadfence_block();
+              sh.heavy_posted = sh.heavy_posted + 1u;
+            }
+          } else if (row_cnt <= p.csr_cap) {
             const uint32_t* list = csr + slot * p.csr_cap;
             for (uint32_t i = lane; i < row_cnt; i += 32) {
               const unsigned long long at = static_cast<unsigned long long>(out_base) + i;
@@ -1247,49 +1358,36 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
               }
             }
           } else {
-            // more outliers than the list holds: take them from the input row in global memory again,
-            // 2048 elements (eight 16-byte loads per lane) per round trip
+            // more outliers than the list holds: the list holds the groups' bitmaps instead.  32 groups per turn:
+            // a scan of the counts, then every lane reads its group's 64 bytes from the input again (one round
+            // trip for the whole turn) and writes its entries
+            const uint32_t* bms = csr + slot * p.csr_cap;
             const uint4* xrow4 = reinterpret_cast<const uint4*>(p.x + static_cast<size_t>(tile) * p.hidden);
             unsigned long long pos = out_base;
-            for (uint32_t c0 = 0; c0 < p.chunks; c0 += 256u) {
-              uint4 v[8];
+            for (uint32_t g0 = 0; g0 < nt; g0 += 32u) {
+              const uint32_t g = g0 + lane;
+              const uint32_t bm = bms[g];
+              const uint32_t cnt = __popc(bm);
+              uint32_t incl = cnt;
 #pragma unroll
-              for (uint32_t k = 0; k < 8u; ++k) {
-                const uint32_t c = c0 + 32u * k + lane;
-                v[k] = c < p.chunks ? xrow4[c] : make_uint4(0u, 0u, 0u, 0u);
+              for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t up = __shfl_up_sync(kFull, incl, d);
+                if (lane >= static_cast<uint32_t>(d)) incl += up;
               }
+              unsigned long long at = pos + (incl - cnt);
+              pos += __shfl_sync(kFull, incl, 31);
+              if (bm != 0u) {
+                uint4 v[4];
 #pragma unroll
-              for (uint32_t k = 0; k < 8u; ++k) {
-                const uint32_t c = c0 + 32u * k + lane;  // this lane's eight elements: 8c .. 8c + 7
-                const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
-                uint32_t raw[8], cnt = 0u;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  raw[j] = (j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xffffu);
-                  // patterns of non-negative values order like the values; NaN patterns sort above +Inf
-                  cnt += (c < p.chunks && (raw[j] & 0x7fffu) >= p.thr16) ? 1u : 0u;
-                }
-                uint32_t incl = cnt;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                  const uint32_t up = __shfl_up_sync(kFull, incl, d);
-                  if (lane >= static_cast<uint32_t>(d)) incl += up;
-                }
-                unsigned long long at = pos + (incl - cnt);
-                pos += __shfl_sync(kFull, incl, 31);
-                if (cnt != 0u) {
-#pragma unroll
-                  for (int j = 0; j < 8; ++j) {
-                    if ((raw[j] & 0x7fffu) >= p.thr16) {
-                      if (at < p.lay.outlier_capacity) {
-                        o_outl[at] = ((8u * c + static_cast<uint32_t>(j)) << 16) | raw[j];
-                      } else {
-                        overflow = true;
-                      }
-                      ++at;
-                    }
+                for (uint32_t j = 0; j < 4; ++j) v[j] = 4u * g + j < p.chunks ? xrow4[4u * g + j] : make_uint4(0u, 0u, 0u, 0u);
+                for_each_flagged(bm, v, 32u * g, [&](uint32_t entry) {
+                  if (at < p.lay.outlier_capacity) {
+                    o_outl[at] = entry;
+                  } else {
+                    overflow = true;
                   }
-                }
+                  ++at;
+                });
               }
             }
           }

@@ -229,6 +229,22 @@ def test_long_rows_with_few_and_very_many_outliers_mixed(dtype):
     full_parity(x, 6.0, [2, 4, 8], 0.2, check_cross=False)
 
 
+@pytest.mark.parametrize("hidden,max_outliers", [(4096, 0), (5120, 0), (1000, 0), (4096, 300000)])
+def test_runs_of_rows_that_are_mostly_outliers(hidden, max_outliers):
+    # every persistent CTA meets several rows in a row whose outliers exceed its lists (a third to all of the row),
+    # between stretches of ordinary rows; the last case also runs out of CSR capacity in the middle of such a row
+    T = 1500
+    g = torch.Generator().manual_seed(hidden)
+    v = torch.randn((T, hidden), generator=g)
+    v[300:900] *= torch.linspace(4.0, 40.0, 600).unsqueeze(1)
+    v[1200:1230] *= 100.0
+    x = v.to(torch.float16).contiguous()
+    counts = (~(x.float().abs() < 6.0)).sum(dim=1)
+    assert int((counts > hidden // 3).sum()) > 500 and int((counts == 0).sum()) > 100
+    gpu_blob, _ = full_parity(x, 6.0, [2, 4, 8], 0.2, max_outliers=max_outliers, check_cross=False)
+    assert R.header(gpu_blob)["status"] == (6 if max_outliers else 0)
+
+
 # ------------------------------------------------------------------ asynchronous conditions and errors
 
 def test_outlier_overflow_is_reported():
