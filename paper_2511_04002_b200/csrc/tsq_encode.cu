@@ -73,23 +73,21 @@ struct __align__(16) Level {
   float r;    // fl(1 / s)
   int zp;     // zero-point rint(m_min / s)
   int qmax;   // 2^(b-1) - 1
-  int plain;  // the fast steps apply: FMA quotient safe, zero-point 0, no code needs the clamp (see the file header)
-  int pad[3];
 };
 
-__device__ __forceinline__ Level make_level(float mmin, float mmax, int b) {
+// *plain: the fast steps apply to the level: FMA quotient safe, zero-point 0, no code needs the clamp (see the file header).
+__device__ __forceinline__ Level make_level(float mmin, float mmax, int b, bool* plain) {
   Level c;
   c.qmax = (1 << (b - 1)) - 1;
   const float range = __fsub_rn(mmax, mmin);
   c.s = range > 0.0f ? __fdiv_rn(range, static_cast<float>(c.qmax)) : (mmax > 0.0f ? mmax : 1.0f);
   c.zp = mmin > 0.0f ? __float2int_rn(__fdiv_rn(mmin, c.s)) : 0;  // 0 / s = 0: the usual row needs no division here
   c.r = __frcp_rn(c.s);
-  c.pad[0] = c.pad[1] = c.pad[2] = 0;
   // Plain: no intermediate of the FMA quotient can leave the normal range, the zero-point is 0 (so no code is
   // negative) and the largest magnitude's code needs no clamp (codes grow with the magnitude).  With a minimum
   // of 0 the scale is fl(max / Qmax) and max / scale rounds to Qmax: no division needed to know.
-  c.plain = ((c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && c.zp == 0 &&
-             (mmin == 0.0f || __float2int_rn(__fdiv_rn(mmax, c.s)) <= c.qmax)) ? 1 : 0;
+  *plain = (c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && c.zp == 0 &&
+           (mmin == 0.0f || __float2int_rn(__fdiv_rn(mmax, c.s)) <= c.qmax);
   return c;
 }
 
@@ -104,8 +102,6 @@ __device__ __forceinline__ Level make_level_signed(float vmin, float vmax, int b
   c.s = range > 0.0f ? __fdiv_rn(range, static_cast<float>(c.qmax)) : (a > 0.0f ? a : 1.0f);
   c.zp = __float2int_rn(__fdiv_rn(vmin, c.s));
   c.r = 0.0f;
-  c.plain = 0;
-  c.pad[0] = c.pad[1] = c.pad[2] = 0;
   return c;
 }
 
@@ -464,14 +460,15 @@ __device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartial
   const uint32_t total = __shfl_sync(kFull, incl, 31);
   // SV: the partial results are order keys of signed values
   const int b = p.bits[min(lane, static_cast<uint32_t>(p.n_bits - 1))];
+  bool plain = false;
   const Level lv = SV ? make_level_signed(E::pattern_f32(pattern_of_key(pmin)), E::pattern_f32(pattern_of_key(pmax)), b)
-                      : make_level(E::pattern_f32(pmin), E::pattern_f32(pmax), b);
+                      : make_level(E::pattern_f32(pmin), E::pattern_f32(pmax), b, &plain);
   if (lane < static_cast<uint32_t>(p.n_bits)) {
     lv_out[lane] = lv;
     S_out[lane] = 0;
   }
   if (lane == 0) *row_cnt = total;
-  return __all_sync(kFull, lv.plain != 0) ? 0u : 1u;
+  return __all_sync(kFull, plain) ? 0u : 1u;
 }
 
 // The limit on device-side waits: the workspace's setting, else the built-in one.
@@ -903,7 +900,7 @@ struct RowMeta {
   uint32_t bstar, agg_w;
   float scale;
   int zp;
-  uint32_t heavy;  // 0, or 1 + the side buffer that holds the row's outlier bitmaps (more outliers than a list holds)
+  uint32_t heavy;  // 1: the side buffer holds the row's outlier bitmaps (more outliers than a list holds)
 };
 
 struct PipeShared {
@@ -918,13 +915,14 @@ struct PipeShared {
                                // compute threads act on, so that all of them leave the row loop in the same iteration
   uint32_t wait_limit;         // polls before a handshake gives up
   uint32_t next_tile[2];       // ticket of the row after the current one, by iteration parity
-  // Rows with more outliers than a ring slot's list holds: the compute threads leave the groups' bitmaps in one of two
-  // side buffers, the placement warp posts the row's CSR offset there once it is resolved, and the compute threads
-  // write the entries themselves, all at once, at the top of a later iteration.
-  uint32_t heavy_bm[2][kPipeMaxThreads - 64];
-  uint32_t heavy_wcnt[2][(kPipeMaxThreads - 64) / 32];  // exclusive scan of the warps' outlier counts
-  uint32_t heavy_tile[2];
-  volatile uint32_t heavy_base[2];   // out_ptr[tile], from the placement warp
+  // Rows with more outliers than a ring slot's list holds: the compute threads leave the groups' bitmaps in a side
+  // buffer, the placement warp posts the row's CSR offset there once it is resolved, and the compute threads write
+  // the entries themselves, all at once, at the top of a later iteration.  (One buffer: a second one would cost
+  // the ring a slot at hidden 8192.  A row that finds it taken leaves its bitmaps in the list instead.)
+  uint32_t heavy_bm[kPipeMaxThreads - 64];
+  uint32_t heavy_wcnt[(kPipeMaxThreads - 64) / 32];  // exclusive scan of the warps' outlier counts
+  uint32_t heavy_tile;
+  volatile uint32_t heavy_base;      // out_ptr[tile], from the placement warp
   volatile uint32_t heavy_posted;    // such rows whose offset has been posted
   volatile uint32_t heavy_seen[2];   // heavy_posted as thread 0 saw it before the iteration's barrier, by iteration parity
 };
@@ -989,13 +987,13 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
     uint32_t n_a = 0u;       // rows of this CTA that finished pass A; n_a - have_prev of them are packed
     uint32_t bitmap_prev = 0u, cnt_prev = 0u, first_prev = 0u;  // outliers of the thread's group in row n_a - 1
     uint32_t slot = 0u;      // ring slot of the next row to be packed: (rows packed so far) mod p.ring
-    uint32_t heavy_filled = 0u, heavy_done = 0u;  // rows put into / written out of the side buffers (the same in every thread)
-    // The CSR entries of the row in side buffer k, to their place in the blob: every thread takes its own group.
-    const auto emit_heavy = [&](uint32_t k) {
-      const uint32_t bm = sh.heavy_bm[k][u];
-      const uint32_t wbase = sh.heavy_wcnt[k][warp];
-      const uint32_t tile_h = sh.heavy_tile[k];
-      const uint32_t base = sh.heavy_base[k];
+    uint32_t heavy_filled = 0u, heavy_done = 0u;  // rows put into / written out of the side buffer (the same in every thread)
+    // The CSR entries of the row in the side buffer, to their place in the blob: every thread takes its own group.
+    const auto emit_heavy = [&]() {
+      const uint32_t bm = sh.heavy_bm[u];
+      const uint32_t wbase = sh.heavy_wcnt[warp];
+      const uint32_t tile_h = sh.heavy_tile;
+      const uint32_t base = sh.heavy_base;
       const uint32_t cnt = __popc(bm);
       uint32_t incl = cnt;
 #pragma unroll
@@ -1086,9 +1084,9 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       }
       compute_barrier(nt);
       if (sh.stop[it & 1u] != 0u) break;
-      const uint32_t heavy_done_before = heavy_done;  // a side buffer emptied in this iteration is refilled in a later one
+      const uint32_t heavy_done_before = heavy_done;  // the side buffer, emptied in this iteration, is refilled in a later one
       if (heavy_done < heavy_filled && sh.heavy_seen[it & 1u] > heavy_done) {
-        emit_heavy(heavy_done & 1u);
+        emit_heavy();
         ++heavy_done;
       }
       if (tid == 0) {
@@ -1194,11 +1192,11 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         const uint32_t row_cnt = m.row_cnt;
         const uint32_t agg_w = static_cast<uint32_t>(bstar) * p.lay.wpp;
         // more outliers than the slot's list holds: into a side buffer when one is free
-        const bool to_heavy = row_cnt > p.csr_cap && heavy_filled - heavy_done_before < 2u;
+        const bool to_heavy = row_cnt > p.csr_cap && heavy_filled == heavy_done_before;
         if (tid == 0) {
           // the row's sizes are known: let the rows behind it see them
           publish_aggregate(p, gen4, tile_prev, agg_w, row_cnt);
-          m.heavy = to_heavy ? 1u + (heavy_filled & 1u) : 0u;
+          m.heavy = to_heavy ? 1u : 0u;
           m.bstar = static_cast<uint32_t>(bstar);
           m.agg_w = agg_w;
           m.scale = m.lv[best_ci].s;
@@ -1215,10 +1213,9 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         //      both are taken, in the list itself (it has room for at least two words per compute thread), where
         //      the placement warp makes the entries from them ----
         if (to_heavy) {
-          const uint32_t k = heavy_filled & 1u;
-          sh.heavy_bm[k][u] = bitmap_prev;
-          if (lane == 0) sh.heavy_wcnt[k][warp] = m.part.warp_cnt[warp];
-          if (tid == 0) sh.heavy_tile[k] = tile_prev;
+          sh.heavy_bm[u] = bitmap_prev;
+          if (lane == 0) sh.heavy_wcnt[warp] = m.part.warp_cnt[warp];
+          if (tid == 0) sh.heavy_tile = tile_prev;
           ++heavy_filled;
         } else if (slot_free && row_cnt > p.csr_cap) {
           csr[slot * p.csr_cap + u] = bitmap_prev;
@@ -1284,7 +1281,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       if (tid == 0) sh.heavy_seen[0] = wait_beyond(&sh.heavy_posted, heavy_done, sh, false, 200u) ? 1u : 0u;
       compute_barrier(nt);
       const bool posted = sh.heavy_seen[0] != 0u;
-      if (posted) emit_heavy(heavy_done & 1u);
+      if (posted) emit_heavy();
       ++heavy_done;
       compute_barrier(nt);  // before thread 0 writes heavy_seen[0] again
       if (!posted) break;   // the CTA aborted
@@ -1343,7 +1340,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           if (m.heavy != 0u) {
             // the compute threads write this row's entries: tell them where
             if (lane == 0) {
-              sh.heavy_base[m.heavy - 1u] = out_base;
+              sh.heavy_base = out_base;
               __threadfence_block();
               sh.heavy_posted = sh.heavy_posted + 1u;
             }
