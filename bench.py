@@ -348,6 +348,10 @@ def other_workloads(B, device, peak):
               synth.c5_sweep_point(4, 1, 0), synth.c5_sweep_point(4, 2, 1)):
         out[w.name] = time_workload(B, device, w, peak)
         torch.cuda.empty_cache()
+    # a KV cache through the same codec (keys and values of 20 layers for 256 tokens)
+    w = synth.kv_cache()
+    out[w.name] = time_workload(B, device, w, peak)
+    torch.cuda.empty_cache()
     # the signed-values variant of the codec (AIQ on the signed inliers, no sign plane) on the c3 tensor
     w = synth.c3_13b_prefill()
     out[w.name + "_signed_values"] = time_workload(B, device, w, peak, variant=B.VARIANT_SIGNED_VALUES)

@@ -32,6 +32,9 @@ class Recipe:
     channel_outliers: Tuple[int, float] = (0, 1.0)   # (number of fixed channels, multiplier)
     random_outliers: Tuple[float, str, float, float] = (0.0, "none", 0.0, 0.0)
     # (rate, kind, p0, p1): kind "absnormal" -> +-|N(p0, p1)|, "uniform" -> +-U(p0, p1)
+    kv_layers: int = 0                   # > 0: a KV cache, rows ordered [layer][key | value][token], tokens = 2 * kv_layers * w:
+                                         # every layer's keys and values get their own factor exp(N(0, 0.3)), and the
+                                         # fixed outlier channels exist in the key rows only
 
 
 @dataclass(frozen=True)
@@ -59,6 +62,15 @@ def generate(recipe: Recipe, seed: int, row_chunk: int = 1024) -> torch.Tensor:
     n_ch, ch_mult = recipe.channel_outliers
     channels = rng.choice(H, size=n_ch, replace=False) if n_ch > 0 else None
     rate, kind, p0, p1 = recipe.random_outliers
+    layer_scale, is_key = None, None
+    if recipe.kv_layers > 0:
+        if T % (2 * recipe.kv_layers) != 0:
+            raise ValueError("a KV cache of %d layers needs a multiple of %d rows" % (recipe.kv_layers, 2 * recipe.kv_layers))
+        w = T // (2 * recipe.kv_layers)
+        factors = np.exp(rng.standard_normal(2 * recipe.kv_layers) * 0.3).astype(np.float32)   # [layer][key | value]
+        block = np.arange(T) // w
+        layer_scale = factors[block][:, None]
+        is_key = (block % 2 == 0)
     for t0 in range(0, T, row_chunk):
         t1 = min(T, t0 + row_chunk)
         n = t1 - t0
@@ -71,8 +83,14 @@ def generate(recipe: Recipe, seed: int, row_chunk: int = 1024) -> torch.Tensor:
         if recipe.token_scale_sigma > 0:
             g = np.exp(rng.standard_normal((n, 1)) * recipe.token_scale_sigma).astype(np.float32)
             v *= g
+        if layer_scale is not None:
+            v *= layer_scale[t0:t1]
         if channels is not None:
-            v[:, channels] *= np.float32(ch_mult)
+            if is_key is None:
+                v[:, channels] *= np.float32(ch_mult)
+            else:
+                rows = np.nonzero(is_key[t0:t1])[0]
+                v[np.ix_(rows, channels)] *= np.float32(ch_mult)
         if rate > 0:
             hit = rng.random((n, H), dtype=np.float32) < np.float32(rate)
             k = int(hit.sum())
@@ -127,6 +145,15 @@ def c4_70b_prefill(tokens: int = 8192) -> Workload:
                     Recipe(tokens, 8192, "bf16", "student_t", nu=3.0,
                            random_outliers=(0.001, "uniform", 20.0, 100.0)),
                     tau=8.0, bits=(2, 4, 8), seed=4)
+
+
+def kv_cache(w: int = 256, layers: int = 20) -> Workload:
+    """Keys and values of the first `layers` decoder layers for w tokens of a 7B-shaped model (4096 = heads x head
+    dimension), the tensor Eq. "bkv" sizes: [2 * layers * w] rows through the same codec."""
+    rows = 2 * layers * w
+    return Workload("kv_llama2_7b_l%d_w%d_%dx4096_f16" % (layers, w, rows),
+                    Recipe(rows, 4096, "f16", "normal", token_scale_sigma=0.2, channel_outliers=(8, 8.0), kv_layers=layers),
+                    tau=6.0, bits=(2, 4, 8), seed=7)
 
 
 C5_TOKENS = (1, 16, 256, 4096, 32768)

@@ -196,6 +196,14 @@ def test_c4_70b_prefill_reduced():
     full_parity(synth.make(w), w.tau, w.bits, w.delta, check_cross=False)
 
 
+@pytest.mark.parametrize("w", [8, 256])
+def test_kv_cache_workload(w):
+    wl = synth.kv_cache(w)
+    x = synth.make(wl)
+    gpu_blob, _ = full_parity(x, wl.tau, wl.bits, wl.delta, check_cross=False)
+    assert R.header(gpu_blob)["total_outliers"] > 0
+
+
 @pytest.mark.parametrize("i_tok", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("i_rate", [0, 1, 2])
 @pytest.mark.parametrize("i_dtype", [0, 1])
