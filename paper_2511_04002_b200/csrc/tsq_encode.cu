@@ -1080,15 +1080,10 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         // The levels and placement warps may raise abort at any moment.  Thread 0 alone samples it, before the
         // barrier, into a word that nobody else writes: every compute thread then takes the same branch.
         sh.stop[it & 1u] = sh.abort;
-        sh.heavy_seen[it & 1u] = sh.heavy_posted;
+        if (heavy_filled != heavy_done) sh.heavy_seen[it & 1u] = sh.heavy_posted;
       }
       compute_barrier(nt);
       if (sh.stop[it & 1u] != 0u) break;
-      const uint32_t heavy_done_before = heavy_done;  // the side buffer, emptied in this iteration, is refilled in a later one
-      if (heavy_done < heavy_filled && sh.heavy_seen[it & 1u] > heavy_done) {
-        emit_heavy();
-        ++heavy_done;
-      }
       if (tid == 0) {
         __threadfence_block();
         if (have_cur) sh.a_ready = n_a + 1u;
@@ -1192,7 +1187,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         const uint32_t row_cnt = m.row_cnt;
         const uint32_t agg_w = static_cast<uint32_t>(bstar) * p.lay.wpp;
         // more outliers than the slot's list holds: into a side buffer when one is free
-        const bool to_heavy = row_cnt > p.csr_cap && heavy_filled == heavy_done_before;
+        const bool to_heavy = row_cnt > p.csr_cap && heavy_filled == heavy_done;
         if (tid == 0) {
           // the row's sizes are known: let the rows behind it see them
           publish_aggregate(p, gen4, tile_prev, agg_w, row_cnt);
@@ -1242,7 +1237,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             uint32_t bm = bitmap_prev;
             list[at++] = ((32u * u + static_cast<uint32_t>(__ffs(bm) - 1)) << 16) | first_prev;
             bm &= bm - 1u;
-            if (__popc(bm) <= 2) {
+            if (__popc(bm) <= 5) {
               while (bm != 0u) {  // further outliers of the group: read from the input again
                 const uint32_t e = 32u * u + static_cast<uint32_t>(__ffs(bm) - 1);
                 bm &= bm - 1u;
@@ -1261,6 +1256,13 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         }
         fence_proxy_async_smem();  // the planes are about to be read by the bulk-copy engine
         slot = slot + 1u == p.ring ? 0u : slot + 1u;
+      }
+      // the row in the side buffer, once the placement warp has posted its offset (as thread 0 saw it before this
+      // iteration's barrier).  Here, after pass C, so that the buffer is not refilled in the iteration that empties it:
+      // the next pass C comes after the next barrier.
+      if (heavy_filled != heavy_done && sh.heavy_seen[it & 1u] > heavy_done) {
+        emit_heavy();
+        ++heavy_done;
       }
       have_prev = have_cur;
       bitmap_prev = bitmap_cur;
