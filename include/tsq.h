@@ -120,8 +120,7 @@ tsq_status_t tsq_plan(tsq_plan_t **out, int device, tsq_dtype_t dtype, int32_t h
 
 /*
  * The same with the variant chosen (TSQ_VARIANT_*; tsq_plan is this call with TSQ_VARIANT_MAGNITUDES).  Any other
- * value is TSQ_ERR_INVALID_ARG.  Every other call takes plans of either variant.  The signed-values variant is
- * served by the one-CTA-per-row encoder at every size and by the division instruction (no fast steps).
+ * value is TSQ_ERR_INVALID_ARG.  Every other call takes plans of either variant.
  */
 tsq_status_t tsq_plan_variant(tsq_plan_t **out, int device, tsq_dtype_t dtype, int32_t hidden, int64_t max_tokens,
                               float tau, const int32_t *bits, int32_t n_bits, float delta, int64_t max_outliers,

@@ -222,23 +222,22 @@ tsq_status_t tsq_plan_variant(tsq_plan_t** out, int device, tsq_dtype_t dtype, i
     p->pipe_smem = 0;
     int base_blocks = 0;
     uint32_t base_ring = 0;
-    // (the signed-values variant has no pipelined kernel: its calls all take the one-CTA-per-row kernel)
-    for (uint32_t per_group = 2u; ok && variant == TSQ_VARIANT_MAGNITUDES && per_group <= 4u && p->pipe_threads <= kPipeMaxThreads;
-         per_group += 2u) {
+    const bool sv = variant == TSQ_VARIANT_SIGNED_VALUES;
+    for (uint32_t per_group = 2u; ok && per_group <= 4u && p->pipe_threads <= kPipeMaxThreads; per_group += 2u) {
       const uint32_t cap = per_group * p->pipe_compute;
       const auto smem_for = [&](uint32_t ring) {
         return 3u * static_cast<size_t>(p->pipe_park) + ring * (static_cast<size_t>(p->pipe_planes) + 4u * static_cast<size_t>(cap));
       };
       if (smem_for(4u) + 8192 > static_cast<size_t>(smem_optin)) break;
       int blocks = 0;
-      ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, p->pipe_threads, smem_for(4u), &blocks) == cudaSuccess;
+      ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, sv, p->pipe_threads, smem_for(4u), &blocks) == cudaSuccess;
       if (!ok || blocks < 1) break;
       // the deepest ring that leaves the number of resident CTAs as it is
       uint32_t ring = 4u;
       for (uint32_t r = static_cast<uint32_t>(kMaxRing); ok && r > 4u; --r) {
         if (smem_for(r) + 8192 > static_cast<size_t>(smem_optin)) continue;
         int b = 0;
-        ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, p->pipe_threads, smem_for(r), &b) == cudaSuccess;
+        ok = encode_pipe_attrs(dtype == TSQ_BF16, p->pipe_full, sv, p->pipe_threads, smem_for(r), &b) == cudaSuccess;
         if (ok && b == blocks) {
           ring = r;
           break;

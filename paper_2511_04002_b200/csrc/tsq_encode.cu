@@ -92,8 +92,10 @@ __device__ __forceinline__ Level make_level(float mmin, float mmax, int b, bool*
 }
 
 // The signed-values variant (Eq. "Proposed" on the signed inliers): Q_max = 2^b - 1, the zero-point may be
-// negative, a constant row takes its own magnitude as the scale.  Never plain: the division instruction does it.
-__device__ __forceinline__ Level make_level_signed(float vmin, float vmax, int b) {
+// negative, a constant row takes its own magnitude as the scale.  *plain: the fast steps apply: the FMA quotient is
+// safe and no code needs a clamp (codes grow with the value, the smallest is 0 by construction, so the largest
+// value's code decides); the zero-point is then subtracted byte-wise, modulo 256.
+__device__ __forceinline__ Level make_level_signed(float vmin, float vmax, int b, bool* plain) {
   Level c;
   c.qmax = (1 << b) - 1;
   // two finite values of opposite sign can lie further apart than binary32 holds: the largest finite value then
@@ -101,7 +103,8 @@ __device__ __forceinline__ Level make_level_signed(float vmin, float vmax, int b
   const float a = fabsf(vmax);
   c.s = range > 0.0f ? __fdiv_rn(range, static_cast<float>(c.qmax)) : (a > 0.0f ? a : 1.0f);
   c.zp = __float2int_rn(__fdiv_rn(vmin, c.s));
-  c.r = 0.0f;
+  c.r = __frcp_rn(c.s);
+  *plain = (c.s >= 0x1p-60f) && (c.s <= 0x1p60f) && (__float2int_rn(__fdiv_rn(vmax, c.s)) - c.zp <= c.qmax);
   return c;
 }
 
@@ -125,11 +128,13 @@ __device__ __forceinline__ uint32_t codes2_divide(uint32_t x, const Level& c) {
 // ---- plain rows: two elements at a time with the packed binary32 instructions (each lane IEEE round-to-nearest-even) ----
 struct Level2 {
   uint64_t r2, ns2;  // {r, r} and {-s, -s}
+  uint32_t zp4;      // signed-values variant: the zero-point modulo 256 in every byte
 };
 __device__ __forceinline__ Level2 make_level2(const Level& c) {
   Level2 l;
   l.r2 = pack2f(c.r, c.r);
   l.ns2 = pack2f(-c.s, -c.s);
+  l.zp4 = (static_cast<uint32_t>(c.zp) & 0xffu) * 0x01010101u;
   return l;
 }
 // Magnitudes of the two elements of a 16-bit pair as packed binary32.
@@ -154,6 +159,36 @@ __device__ __forceinline__ uint32_t bytes4(uint64_t ta, uint64_t tb) {
   unpack2u(ta, alo, ahi);
   unpack2u(tb, blo, bhi);
   return __byte_perm(mad_u32(blo, 256u, alo), mad_u32(bhi, 256u, ahi), 0x5410);
+}
+
+// 2^23 rounds a non-negative quotient to an integer; 2^23 + 2^22 does the same for |quotient| < 2^22 of either sign
+// and leaves the integer, modulo 2^22, in the low bits of the pattern (two's complement).
+constexpr float kRoundMagicSigned = 12582912.0f;
+// The signed values of the two elements of a 16-bit pair as packed binary32 (signed-values variant).
+template <bool BF16>
+__device__ __forceinline__ uint64_t values2(uint32_t x) {
+  if (BF16) return pack2u(mad_u32(x, 65536u, 0u), x & 0xffff0000u);
+  const float2 f = __half22float2(Elem<false>::as2(x));
+  return pack2f(f.x, f.y);
+}
+// Low bytes of four patterns as one word (bytes a.lo, b.lo, a.hi, b.hi) when the patterns' other bytes are not
+// zero (a negative rounded quotient): byte permutes only.
+__device__ __forceinline__ uint32_t bytes4_any(uint64_t ta, uint64_t tb) {
+  uint32_t alo, ahi, blo, bhi;
+  unpack2u(ta, alo, ahi);
+  unpack2u(tb, blo, bhi);
+  return __byte_perm(__byte_perm(alo, blo, 0x0040), __byte_perm(ahi, bhi, 0x0040), 0x5410);
+}
+// The codes of four elements (pairs xa, xb) at level l as bytes a.lo, b.lo, a.hi, b.hi.  SV: of the signed values,
+// zero-point subtracted modulo 256 (exact for a plain level: every code lies in [0, 255]).
+template <bool BF16, bool SV>
+__device__ __forceinline__ uint32_t codes4(uint32_t xa, uint32_t xb, const Level2& l) {
+  if (SV) {
+    const uint64_t magic2 = pack2f(kRoundMagicSigned, kRoundMagicSigned);
+    return __vsub4(bytes4_any(quotient2(values2<BF16>(xa), l, magic2), quotient2(values2<BF16>(xb), l, magic2)), l.zp4);
+  }
+  const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
+  return bytes4(quotient2(magnitudes2<BF16>(xa), l, magic2), quotient2(magnitudes2<BF16>(xb), l, magic2));
 }
 
 __device__ __forceinline__ uint32_t max_s16x2(uint32_t a, uint32_t b) {
@@ -201,13 +236,21 @@ __device__ __forceinline__ uint32_t split_group(uint32_t (&x)[16], uint32_t nval
 // Pass B on one group of a plain row: sum |(q0 >> sh) - q| over its 32 elements (Algorithm 1's distortion
 // numerator).  Four codes travel as the bytes of one word: the shift and mask take four at a time, and the
 // byte-wise sum-of-absolute-differences instruction adds the four differences.
-template <bool BF16>
-__device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], const Level2& top, const Level2& low, int sh) {
-  const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+// SV (signed-values variant): 8-bit codes of the signed values; the chunks at and past `nvalid` lie beyond the end
+// of the row and do not count (their zeros would get the code of the value 0, which is not 0 there).
+template <bool BF16, bool SV = false>
+__device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], const Level2& top, const Level2& low, int sh,
+                                                     uint32_t nvalid = 4u) {
+  const uint32_t shmask = ((SV ? 0xffu : 0x7fu) >> sh) * 0x01010101u;
   const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
   uint32_t S = 0;
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
+    if (SV) {
+      if (static_cast<uint32_t>(i / 4) >= nvalid) continue;
+      S = __vsadu4((codes4<BF16, true>(x[i], x[i + 1], top) >> sh) & shmask, codes4<BF16, true>(x[i], x[i + 1], low)) + S;
+      continue;
+    }
     const uint64_t ma = magnitudes2<BF16>(x[i]), mb = magnitudes2<BF16>(x[i + 1]);
     const uint32_t ct4 = bytes4(quotient2(ma, top, magic2), quotient2(mb, top, magic2));
     const uint32_t q4 = bytes4(quotient2(ma, low, magic2), quotient2(mb, low, magic2));
@@ -221,17 +264,27 @@ __device__ __forceinline__ uint32_t distortion_group(const uint32_t (&x)[16], co
 // of chunks 2h and 2h + 1, low elements first) and ql the candidate's own codes in the same grouping, no signs.
 // (Any grouping of four serves the sum; this one costs the byte assembly least, and two byte permutes per i
 // turn it into the input of the bit transpose.)
-template <bool BF16>
+// SV: bytes are the 8-bit codes of the signed values, no signs; bytes of chunks at and past `nvalid` are 0.
+template <bool BF16, bool SV = false>
 __device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], const Level2& top, const Level2& low, int sh,
-                                                     uint32_t (&tb)[8], uint32_t (&ql)[8]) {
-  const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+                                                     uint32_t (&tb)[8], uint32_t (&ql)[8], uint32_t nvalid = 4u) {
+  const uint32_t shmask = ((SV ? 0xffu : 0x7fu) >> sh) * 0x01010101u;
   const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
   uint32_t S = 0;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
+    // bytes 0 and 2 of a word belong to chunk 2h, bytes 1 and 3 to chunk 2h + 1
+    const uint32_t inside = (2u * h < nvalid ? 0x00ff00ffu : 0u) | (2u * h + 1u < nvalid ? 0xff00ff00u : 0u);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint32_t xa = x[8 * h + i], xb = x[8 * h + 4 + i];  // pairs i of chunks 2h and 2h + 1
+      if (SV) {
+        const uint32_t ct4 = codes4<BF16, true>(xa, xb, top) & inside, q4 = codes4<BF16, true>(xa, xb, low) & inside;
+        S = __vsadu4((ct4 >> sh) & shmask, q4) + S;
+        tb[4 * h + i] = ct4;
+        ql[4 * h + i] = q4;
+        continue;
+      }
       const uint64_t ma = magnitudes2<BF16>(xa), mb = magnitudes2<BF16>(xb);
       const uint32_t ct4 = bytes4(quotient2(ma, top, magic2), quotient2(mb, top, magic2));
       const uint32_t q4 = bytes4(quotient2(ma, low, magic2), quotient2(mb, low, magic2));
@@ -244,18 +297,25 @@ __device__ __forceinline__ uint32_t distortion_first(const uint32_t (&x)[16], co
 }
 
 // Pass B for a further candidate: the top-level codes come from the bytes the first turn left.
-template <bool BF16>
+template <bool BF16, bool SV = false>
 __device__ __forceinline__ uint32_t distortion_next(const uint32_t (&x)[16], const uint32_t (&tb)[8], const Level2& low, int sh,
-                                                    uint32_t (&ql)[8]) {
-  // a byte of tb is code | sign << 7: shifted right by sh >= 1, the sign bit and the bits that come in from
-  // the next byte all land above the mask
-  const uint32_t shmask = (0x7fu >> sh) * 0x01010101u;
+                                                    uint32_t (&ql)[8], uint32_t nvalid = 4u) {
+  // a byte of tb is code | sign << 7 (SV: an 8-bit code): shifted right by sh >= 1, the sign bit and the bits that
+  // come in from the next byte all land above the mask
+  const uint32_t shmask = ((SV ? 0xffu : 0x7fu) >> sh) * 0x01010101u;
   const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
   uint32_t S = 0;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
+    const uint32_t inside = (2u * h < nvalid ? 0x00ff00ffu : 0u) | (2u * h + 1u < nvalid ? 0xff00ff00u : 0u);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
+      if (SV) {
+        const uint32_t q4 = codes4<BF16, true>(x[8 * h + i], x[8 * h + 4 + i], low) & inside;
+        S = __vsadu4((tb[4 * h + i] >> sh) & shmask, q4) + S;
+        ql[4 * h + i] = q4;
+        continue;
+      }
       const uint32_t q4 = bytes4(quotient2(magnitudes2<BF16>(x[8 * h + i]), low, magic2),
                                  quotient2(magnitudes2<BF16>(x[8 * h + 4 + i]), low, magic2));
       S = __vsadu4((tb[4 * h + i] >> sh) & shmask, q4) + S;
@@ -278,15 +338,20 @@ __device__ __forceinline__ void planes_of_bytes(const uint32_t (&tb)[8], uint32_
 
 // Pass C on one group of a row whose chosen level is plain: codes as bytes (code | sign << 7), transposed into
 // bit-planes: on return r[k] = bit k of every byte, k < 7 code bits, k = 7 signs.
-template <bool BF16>
-__device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level2& lv, uint32_t (&r)[8]) {
+template <bool BF16, bool SV = false>
+__device__ __forceinline__ void pack_group(const uint32_t (&x)[16], const Level2& lv, uint32_t (&r)[8], uint32_t nvalid = 4u) {
   const uint64_t magic2 = pack2f(kRoundMagic, kRoundMagic);
   uint32_t tb[8];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
+    const uint32_t inside = (2u * h < nvalid ? 0x00ff00ffu : 0u) | (2u * h + 1u < nvalid ? 0xff00ff00u : 0u);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint32_t xa = x[8 * h + i], xb = x[8 * h + 4 + i];
+      if (SV) {
+        tb[4 * h + i] = codes4<BF16, true>(xa, xb, lv) & inside;
+        continue;
+      }
       const uint32_t c4 = bytes4(quotient2(magnitudes2<BF16>(xa), lv, magic2), quotient2(magnitudes2<BF16>(xb), lv, magic2));
       tb[4 * h + i] = c4 | (__byte_perm(xa, xb, 0x7351) & 0x80808080u);
     }
@@ -332,27 +397,30 @@ __device__ __forceinline__ void divide_pack_regs(const uint32_t (&x)[16], const 
 // The same two steps for rows that need the division instruction, written as loops over the parked
 // row's words (xw: the row as 32-bit words) so that they take little room in the instruction stream.
 __device__ __forceinline__ uint32_t park_index(uint32_t nt, uint32_t u, uint32_t j);
-template <bool BF16>
-__device__ __noinline__ uint32_t rolled_distortion(const uint32_t* xw, uint32_t nt, uint32_t u, Level top, Level low, int sh) {
+// (SV: only the first `pairs` words, the ones inside the row, count: see divide_distortion_regs.)
+template <bool BF16, bool SV = false>
+__device__ __noinline__ uint32_t rolled_distortion(const uint32_t* xw, uint32_t nt, uint32_t u, Level top, Level low, int sh,
+                                                   uint32_t pairs = 16u) {
   const uint32_t shmask = (0xffffu >> sh) * 0x10001u;
   uint32_t S = 0;
 #pragma unroll 1
-  for (uint32_t i = 0; i < 16; ++i) {
+  for (uint32_t i = 0; i < (SV ? pairs : 16u); ++i) {
     const uint32_t x = xw[4u * park_index(nt, u, i >> 2) + (i & 3u)];
-    const uint32_t a = (codes2_divide<BF16>(x, top) >> sh) & shmask;
-    const uint32_t q = codes2_divide<BF16>(x, low);
+    const uint32_t a = (codes2_divide<BF16, SV>(x, top) >> sh) & shmask;
+    const uint32_t q = codes2_divide<BF16, SV>(x, low);
     const uint32_t d = max_s16x2(a, q) - min_s16x2(a, q);
     S += (d & 0xffffu) + (d >> 16);
   }
   return S;
 }
-template <bool BF16>
-__device__ __noinline__ Planes8 rolled_pack(const uint32_t* xw, uint32_t nt, uint32_t u, Level lv) {
-  uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // r[k] bit e = bit k of the byte (code | sign << 7) of element e
+template <bool BF16, bool SV = false>
+__device__ __noinline__ Planes8 rolled_pack(const uint32_t* xw, uint32_t nt, uint32_t u, Level lv, uint32_t pairs = 16u) {
+  uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // r[k] bit e = bit k of the byte (code | sign << 7; SV: the 8-bit code) of element e
 #pragma unroll 1
-  for (uint32_t i = 0; i < 16; ++i) {
+  for (uint32_t i = 0; i < (SV ? pairs : 16u); ++i) {
     const uint32_t x = xw[4u * park_index(nt, u, i >> 2) + (i & 3u)];
-    const uint32_t b2 = codes2_divide<BF16>(x, lv) | ((x >> 8) & 0x00800080u);  // elements 2i (byte 0) and 2i + 1 (byte 2)
+    // elements 2i (byte 0) and 2i + 1 (byte 2)
+    const uint32_t b2 = codes2_divide<BF16, SV>(x, lv) | (SV ? 0u : ((x >> 8) & 0x00800080u));
 #pragma unroll
     for (int k = 0; k < 8; ++k) r[k] |= (((b2 >> k) & 1u) << (2u * i)) | (((b2 >> (16 + k)) & 1u) << (2u * i + 1u));
   }
@@ -461,7 +529,7 @@ __device__ __forceinline__ uint32_t row_levels(const EncodeParams& p, RowPartial
   // SV: the partial results are order keys of signed values
   const int b = p.bits[min(lane, static_cast<uint32_t>(p.n_bits - 1))];
   bool plain = false;
-  const Level lv = SV ? make_level_signed(E::pattern_f32(pattern_of_key(pmin)), E::pattern_f32(pattern_of_key(pmax)), b)
+  const Level lv = SV ? make_level_signed(E::pattern_f32(pattern_of_key(pmin)), E::pattern_f32(pattern_of_key(pmax)), b, &plain)
                       : make_level(E::pattern_f32(pmin), E::pattern_f32(pmax), b, &plain);
   if (lane < static_cast<uint32_t>(p.n_bits)) {
     lv_out[lane] = lv;
@@ -677,8 +745,7 @@ struct RowShared {
 };
 
 // MAXT: the largest CTA the instance is launched with (rows of up to 8192 elements get the 256-thread instance,
-// which may use four times the registers of the 1024-thread one).  SV: the signed-values variant, which this
-// kernel alone serves, with the division instruction throughout.
+// which may use four times the registers of the 1024-thread one).  SV: the signed-values variant.
 template <bool BF16, int UPT, int MAXT, bool SV>
 __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(const EncodeParams p) {
   using E = Elem<BF16>;
@@ -758,7 +825,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(
       if (lane == 0) sh.divide = divide;
     }
     __syncthreads();
-    const bool divide = SV || sh.divide != 0u;
+    const bool divide = sh.divide != 0u;
 
     // ---- Algorithm 1: descend the candidate list while the distortion stays within tolerance ----
     const Level top = sh.lv[p.n_bits - 1];
@@ -770,12 +837,10 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(
       uint32_t S = 0;
 #pragma unroll
       for (int k = 0; k < UPT; ++k) {
-        if (SV) {
-          S += divide_distortion_regs<BF16, true>(x[k], top, low, shn, 4u * nvalid[k]);
-        } else if (divide) {
-          S += divide_distortion_regs<BF16>(x[k], top, low, shn);
+        if (divide) {
+          S += divide_distortion_regs<BF16, SV>(x[k], top, low, shn, 4u * nvalid[k]);
         } else {
-          S += distortion_group<BF16>(x[k], make_level2(top), make_level2(low), shn);
+          S += distortion_group<BF16, SV>(x[k], make_level2(top), make_level2(low), shn, nvalid[k]);
         }
       }
       S = __reduce_add_sync(kFull, S);
@@ -793,17 +858,15 @@ __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 2 : 1) encode_rows_kernel(
     uint32_t r[UPT][8];
 #pragma unroll
     for (int k = 0; k < UPT; ++k) {
-      if (SV) {
-        divide_pack_regs<BF16, true>(x[k], best, r[k]);
-        if (nvalid[k] < 4u) {  // pad bits stay 0: the zeros past the end of the row got the code of the value 0
+      if (divide) {
+        divide_pack_regs<BF16, SV>(x[k], best, r[k]);
+        if (SV && nvalid[k] < 4u) {  // pad bits stay 0: the zeros past the end of the row got the code of the value 0
           const uint32_t inside = (1u << (8u * nvalid[k])) - 1u;
 #pragma unroll
           for (int q = 0; q < 8; ++q) r[k][q] &= inside;
         }
-      } else if (divide) {
-        divide_pack_regs<BF16>(x[k], best, r[k]);
       } else {
-        pack_group<BF16>(x[k], make_level2(best), r[k]);
+        pack_group<BF16, SV>(x[k], make_level2(best), r[k], nvalid[k]);
       }
     }
 
@@ -949,7 +1012,8 @@ __device__ __forceinline__ bool wait_beyond(volatile uint32_t* counter, uint32_t
 
 // FULL: every compute thread owns a whole 32-element group (hidden is a multiple of 1024), so none of the
 // checks for short or missing groups is needed.
-template <bool BF16, bool FULL, int MAXT, int MINB>
+// SV: the signed-values variant.
+template <bool BF16, bool FULL, int MAXT, int MINB, bool SV>
 __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodeParams p) {
   using E = Elem<BF16>;
   extern __shared__ __align__(128) unsigned char smem_dyn[];
@@ -1049,6 +1113,19 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         }
         bitmap_cur = split_group<BF16>(x, nvalid, p.thr16 * 0x10001u, mn2, mx2);
         cnt_cur = __popc(bitmap_cur);
+        if (SV) {
+          // min / max of the signed values of T_below instead (outlier slots are +0 by now): as order keys
+          mn2 = 0xffffffffu;
+          mx2 = 0u;
+#pragma unroll
+          for (uint32_t i = 0; i < 16; ++i) {
+            if (FULL || (i >> 2) < nvalid) {
+              const uint32_t key2 = order_keys2(x[i]);
+              mn2 = __vminu2(mn2, key2);
+              mx2 = __vmaxu2(mx2, key2);
+            }
+          }
+        }
         if (bitmap_cur != 0u) {
           // the original pattern of the group's first outlier, from the parked row while it still holds it:
           // the CSR entry is written an iteration later, and most groups with an outlier have just one
@@ -1110,7 +1187,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
           const uint32_t* xw = reinterpret_cast<const uint32_t*>(xp);
           for (int ci = p.n_bits - 2; ci >= 0; --ci) {
             const Level low = m.lv[ci];
-            uint32_t S = rolled_distortion<BF16>(xw, nt, u, top, low, bmax - p.bits[ci]);
+            uint32_t S = rolled_distortion<BF16, SV>(xw, nt, u, top, low, bmax - p.bits[ci], 4u * (FULL ? 4u : group_chunks(p, u)));
             S = __reduce_add_sync(kFull, S);
             if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
             compute_barrier(nt);
@@ -1118,7 +1195,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             bstar = p.bits[ci];
             best_ci = ci;
           }
-          const Planes8 pl = rolled_pack<BF16>(xw, nt, u, m.lv[best_ci]);
+          const Planes8 pl = rolled_pack<BF16, SV>(xw, nt, u, m.lv[best_ci], 4u * (FULL ? 4u : group_chunks(p, u)));
 #pragma unroll
           for (int k = 0; k < 8; ++k) r[k] = pl.v[k];
         } else {
@@ -1140,7 +1217,8 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             }
             const int c0 = ci >= 0 ? ci : 0;
             const Level low = m.lv[c0];
-            uint32_t S = distortion_first<BF16>(y, make_level2(top), make_level2(low), bmax - p.bits[c0], tb, lb);
+            uint32_t S = distortion_first<BF16, SV>(y, make_level2(top), make_level2(low), bmax - p.bits[c0], tb, lb,
+                                                    (FULL || !SV) ? 4u : group_chunks(p, u));
             if (ci >= 0) {
               S = __reduce_add_sync(kFull, S);
               if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
@@ -1168,7 +1246,8 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
                 y[4 * j + 3] = c.w;
               }
               const Level low = m.lv[ci];
-              uint32_t S = distortion_next<BF16>(y, tb, make_level2(low), bmax - p.bits[ci], ql);
+              uint32_t S = distortion_next<BF16, SV>(y, tb, make_level2(low), bmax - p.bits[ci], ql,
+                                                     (FULL || !SV) ? 4u : group_chunks(p, u));
               S = __reduce_add_sync(kFull, S);
               if (lane == 0 && S != 0u) atomicAdd(&m.S[ci], static_cast<int>(S));
               compute_barrier(nt);
@@ -1180,7 +1259,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
             }
             // the chosen candidate's codes with the signs of the top-level bytes
 #pragma unroll
-            for (int k = 0; k < 8; ++k) tb[k] = lb[k] | (tb[k] & 0x80808080u);
+            for (int k = 0; k < 8; ++k) tb[k] = SV ? lb[k] : (lb[k] | (tb[k] & 0x80808080u));
             planes_of_bytes(tb, r);
           }
         }
@@ -1203,7 +1282,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         //      for this row's sizes on top of its own wait. ----
         const bool slot_free = n < p.ring || wait_beyond(&sh.placed, n - p.ring, sh, false, 100u);
         // ---- planes of the chosen level into the row's slot, in blob order ----
-        if (slot_free && (FULL || u < p.units)) store_planes(planes + slot * (p.planes_stride / 4u) + u * static_cast<uint32_t>(bstar), r, bstar, true);
+        if (slot_free && (FULL || u < p.units)) store_planes<SV>(planes + slot * (p.planes_stride / 4u) + u * static_cast<uint32_t>(bstar), r, bstar, true);
         // ---- a row with more outliers than the list holds leaves its groups' bitmaps in a side buffer, or, when
         //      both are taken, in the list itself (it has room for at least two words per compute thread), where
         //      the placement warp makes the entries from them ----
@@ -1294,7 +1373,7 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       if (!wait_beyond(&sh.a_ready, n, sh, true, 500u)) break;
       __threadfence_block();
       RowMeta& m = sh.meta[n % kMetaRing];
-      const uint32_t divide = row_levels<BF16>(p, m.part, nwarps, lane, m.lv, m.S, &m.row_cnt);
+      const uint32_t divide = row_levels<BF16, (kPipeMaxThreads - 64) / 32, SV>(p, m.part, nwarps, lane, m.lv, m.S, &m.row_cnt);
       if (lane == 0) m.divide = divide;
       __syncwarp();
       if (lane == 0) {
@@ -1419,50 +1498,62 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
 
 // The pipelined kernel is built for CTAs of up to kPipeMaxThreads threads (rows of up to 8192 elements)
 // and may use up to 102 registers per thread; longer rows take encode_rows_kernel.
-static const void* pipe_kernel(bool bf16, bool full) {
+template <bool SV>
+static const void* pipe_kernel_of(bool bf16, bool full) {
   if (full) {
-    return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, true, kPipeMaxThreads, 2>)
-                : reinterpret_cast<const void*>(&encode_pipe_kernel<false, true, kPipeMaxThreads, 2>);
+    return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, true, kPipeMaxThreads, 2, SV>)
+                : reinterpret_cast<const void*>(&encode_pipe_kernel<false, true, kPipeMaxThreads, 2, SV>);
   }
-  return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, false, kPipeMaxThreads, 2>)
-              : reinterpret_cast<const void*>(&encode_pipe_kernel<false, false, kPipeMaxThreads, 2>);
+  return bf16 ? reinterpret_cast<const void*>(&encode_pipe_kernel<true, false, kPipeMaxThreads, 2, SV>)
+              : reinterpret_cast<const void*>(&encode_pipe_kernel<false, false, kPipeMaxThreads, 2, SV>);
 }
+static const void* pipe_kernel(bool bf16, bool full, bool sv) { return sv ? pipe_kernel_of<true>(bf16, full) : pipe_kernel_of<false>(bf16, full); }
 
-cudaError_t encode_pipe_attrs(bool bf16, bool full, int threads, size_t smem, int* blocks_per_sm) {
+cudaError_t encode_pipe_attrs(bool bf16, bool full, bool sv, int threads, size_t smem, int* blocks_per_sm) {
   if (threads > kPipeMaxThreads) return cudaErrorInvalidValue;
-  const void* fn = pipe_kernel(bf16, full);
+  const void* fn = pipe_kernel(bf16, full, sv);
   // the attribute belongs to the kernel on the current device, not to a plan: it only ever grows, so
   // that every plan can launch
   static std::mutex mu;
-  static size_t granted[kMaxDevices][2][2] = {};
+  static size_t granted[kMaxDevices][2][2][2] = {};
   {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(mu);
-    if (smem > granted[dev][bf16 ? 1 : 0][full ? 1 : 0]) {
+    size_t& have = granted[dev][bf16 ? 1 : 0][full ? 1 : 0][sv ? 1 : 0];
+    if (smem > have) {
       e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      granted[dev][bf16 ? 1 : 0][full ? 1 : 0] = smem;
+      have = smem;
     }
   }
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads, smem);
 }
 
-cudaError_t launch_encode_pipe(const EncodeParams& p, bool full, int grid, int threads, size_t smem, cudaStream_t stream) {
-  if (threads > kPipeMaxThreads) return cudaErrorInvalidValue;
+template <bool SV>
+static void launch_pipe_variant(const EncodeParams& p, bool full, int grid, int threads, size_t smem, cudaStream_t stream) {
   const bool bf16 = p.dtype == TSQ_BF16;
   if (full) {
     if (bf16) {
-      encode_pipe_kernel<true, true, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
+      encode_pipe_kernel<true, true, kPipeMaxThreads, 2, SV><<<grid, threads, smem, stream>>>(p);
     } else {
-      encode_pipe_kernel<false, true, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
+      encode_pipe_kernel<false, true, kPipeMaxThreads, 2, SV><<<grid, threads, smem, stream>>>(p);
     }
   } else if (bf16) {
-    encode_pipe_kernel<true, false, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
+    encode_pipe_kernel<true, false, kPipeMaxThreads, 2, SV><<<grid, threads, smem, stream>>>(p);
   } else {
-    encode_pipe_kernel<false, false, kPipeMaxThreads, 2><<<grid, threads, smem, stream>>>(p);
+    encode_pipe_kernel<false, false, kPipeMaxThreads, 2, SV><<<grid, threads, smem, stream>>>(p);
+  }
+}
+
+cudaError_t launch_encode_pipe(const EncodeParams& p, bool full, int grid, int threads, size_t smem, cudaStream_t stream) {
+  if (threads > kPipeMaxThreads) return cudaErrorInvalidValue;
+  if (p.variant != 0u) {
+    launch_pipe_variant<true>(p, full, grid, threads, smem, stream);
+  } else {
+    launch_pipe_variant<false>(p, full, grid, threads, smem, stream);
   }
   return cudaGetLastError();
 }

@@ -91,7 +91,7 @@ struct EncodeParams {
   // pipelined kernel only: thread split, shared-memory strides (bytes; csr_cap in entries), ring depth in rows
   uint32_t compute_threads, park_stride, planes_stride, csr_cap, ring;
   uint32_t dtype;
-  uint32_t variant;                          // 0: sign + magnitude codes; 1: codes of the signed values (one-CTA-per-row kernel only)
+  uint32_t variant;                          // 0: sign + magnitude codes; 1: codes of the signed values
   float tau, delta;
 };
 
@@ -108,7 +108,7 @@ struct DecodeParams {
 
 cudaError_t launch_encode_rows(const EncodeParams& p, int grid, int threads, int groups_per_thread, cudaStream_t stream);
 cudaError_t launch_encode_pipe(const EncodeParams& p, bool full, int grid, int threads, size_t smem, cudaStream_t stream);
-cudaError_t encode_pipe_attrs(bool bf16, bool full, int threads, size_t smem, int* blocks_per_sm);
+cudaError_t encode_pipe_attrs(bool bf16, bool full, bool signed_values, int threads, size_t smem, int* blocks_per_sm);
 cudaError_t launch_decode(const DecodeParams& p, int grid, int threads, size_t smem, cudaStream_t stream);
 cudaError_t decode_kernel_attrs(bool bf16, int threads, size_t smem, int* blocks_per_sm);
 size_t decode_smem_bytes(uint32_t row_bytes);

@@ -101,6 +101,20 @@ def test_c1_and_c3_workloads():
         full_parity(synth.make(w), w.tau, w.bits, w.delta, check_cross=False, variant=SV)
 
 
+def test_runs_of_rows_that_are_mostly_outliers():
+    # rows whose outliers exceed a persistent CTA's lists, several in a row, between stretches of ordinary rows
+    T, H = 1200, 4096
+    g = torch.Generator().manual_seed(4096)
+    v = torch.randn((T, H), generator=g)
+    v[300:800] *= torch.linspace(4.0, 40.0, 500).unsqueeze(1)
+    full_parity(v.to(torch.bfloat16).contiguous(), 6.0, [2, 4, 8], 0.2, check_cross=False, variant=SV)
+
+
+def test_c4_shaped_rows():
+    w = synth.c4_70b_prefill(1024)
+    full_parity(synth.make(w), w.tau, w.bits, w.delta, check_cross=False, variant=SV)
+
+
 def test_outlier_overflow_is_reported():
     x = rand16((40, 512), torch.float16, seed=77, scale=3.0, outlier_rate=0.05)
     raw = synth.raw_u16(x)
