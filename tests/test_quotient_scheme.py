@@ -77,3 +77,50 @@ def test_fma_quotient_equals_the_ieee_quotient_after_rint(bf16):
             dense = range(max(1, pmax - 3 * step), pmax + 1)
             sparse = rng.integers(1, max(2, pmax - 3 * step), 200).tolist() if pmax > 3 * step + 2 else []
             check_row(pmax, bf16, b, list(dense) + sparse)
+
+
+def check_signed_row(pmin: int, pmax: int, bf16: bool, b: int, patterns) -> int:
+    """The signed-values variant's fast steps on a row that spans [-value(pmin), +value(pmax)]: the same three
+    operations on the signed value, rounding by adding 2^23 + 2^22, the code as the low byte of the sum's integer
+    minus the zero-point, modulo 256.  Returns how many patterns were checked (rows that are not plain: 0)."""
+    qmax = (1 << b) - 1
+    vmin, vmax = -pattern_value(pmin, bf16), pattern_value(pmax, bf16)
+    s = f32(f32(vmax - vmin) / qmax)
+    r = f32(1 / s)
+    zp = rint(f32_signed(vmin / s))
+    if rint(f32_signed(vmax / s)) - zp > qmax:
+        return 0                                        # a code would need the clamp: such a level takes the division instruction
+    magic = Fraction(12582912)
+    n = 0
+    for sign, bound in ((1, pmax), (-1, pmin)):
+        for p in patterns:
+            if p > bound:
+                continue
+            v = sign * pattern_value(p, bf16)
+            want = rint(f32_signed(v / s)) - zp
+            assert 0 <= want <= qmax
+            q0 = f32_signed(v * r)
+            e = f32_signed(v - q0 * s)
+            q = f32_signed(q0 + e * r)
+            t = f32_signed(q + magic)
+            assert t.denominator == 1 and Fraction(2) ** 23 <= t < Fraction(2) ** 24
+            low22 = (int(t) - (1 << 23)) & 0x3fffff        # the pattern's low mantissa bits: 2^22 + k
+            assert ((low22 & 0xff) - (zp & 0xff)) & 0xff == want, (pmin, pmax, bf16, b, sign, p)
+            n += 1
+    return n
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_signed_values_fast_steps(bf16):
+    rng = np.random.default_rng(17 if bf16 else 19)
+    lo, hi = (0x3c00, 0x4600) if bf16 else (0x3000, 0x5000)
+    checked = 0
+    for _ in range(10):
+        pmin, pmax = int(rng.integers(lo, hi)), int(rng.integers(lo, hi))
+        for b in (2, 4, 8):
+            top = max(pmin, pmax)
+            step = 0x80 if bf16 else 0x400
+            dense = list(range(max(1, top - 2 * step), top + 1))
+            sparse = rng.integers(0, max(2, top - 2 * step), 150).tolist()
+            checked += check_signed_row(pmin, pmax, bf16, b, dense + sparse)
+    assert checked > 5000
