@@ -1389,6 +1389,29 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
       __threadfence_block();
       const RowMeta& m = sh.meta[n % kMetaRing];
       const uint32_t tile = m.tile, agg_w = m.agg_w, row_cnt = m.row_cnt;
+      // Everything the stores below need from shared memory is read before the look-back, whose round trips it then
+      // overlaps with: the token's fields (one per lane: a lone warp pays for every divergent branch, so each lane
+      // selects its field's address and value and one store serves them all) and, for the usual row, whose CSR
+      // entries number 64 at most, the entries themselves, two per lane.
+      const uint32_t heavy = m.heavy;
+      const bool short_list = heavy == 0u && row_cnt <= 64u && row_cnt <= p.csr_cap;
+      uint32_t e0 = 0u, e1 = 0u;
+      if (short_list) {
+        const uint32_t* list = csr + slot * p.csr_cap;
+        if (lane < row_cnt) e0 = list[lane];
+        if (lane + 32u < row_cnt) e1 = list[lane + 32u];
+      }
+      // lanes 1 .. 4: scale, zero-point, word_off[tile + 1], out_ptr[tile + 1]; lanes 5, 6 (first token only): the two leading zeros
+      unsigned long long field_off = 0ull;
+      uint32_t field_val = 0u;
+      bool field = false;
+      if (lane == 1u) { field_off = p.lay.off_scale + 4ull * tile; field_val = __float_as_uint(m.scale); field = true; }
+      if (lane == 2u) { field_off = p.lay.off_zp + 4ull * tile; field_val = static_cast<uint32_t>(m.zp); field = true; }
+      if (lane == 3u) { field_off = p.lay.off_word_off + 4ull * (tile + 1u); field_val = agg_w; field = true; }
+      if (lane == 4u) { field_off = p.lay.off_out_ptr + 4ull * (tile + 1u); field_val = row_cnt; field = true; }
+      if (lane == 5u && tile == 0u) { field_off = p.lay.off_word_off; field = true; }
+      if (lane == 6u && tile == 0u) { field_off = p.lay.off_out_ptr; field = true; }
+      const uint32_t bstar8 = m.bstar;
       uint32_t word_off = 0, out_base = 0;
       const int st = resolve_prefix<1>(p, gen4, tile, agg_w, row_cnt, lane, &word_off, &out_base, lookback_limit(p));
       if (st != TSQ_OK) {
@@ -1407,18 +1430,31 @@ __global__ void __launch_bounds__(MAXT, MINB) encode_pipe_kernel(const EncodePar
         } else {  // runs of words that are not multiples of 16 bytes: plain stores
           for (uint32_t w = lane; w < agg_w; w += 32) wdst[w] = src[w];
         }
-        // the token's fields, one lane each
-        if (lane == 0) reinterpret_cast<uint8_t*>(p.blob + p.lay.off_bits)[tile] = static_cast<uint8_t>(m.bstar);
-        if (lane == 1) reinterpret_cast<float*>(p.blob + p.lay.off_scale)[tile] = m.scale;
-        if (lane == 2) reinterpret_cast<int32_t*>(p.blob + p.lay.off_zp)[tile] = m.zp;
-        if (lane == 3) reinterpret_cast<uint32_t*>(p.blob + p.lay.off_word_off)[tile + 1u] = word_off + agg_w;
-        if (lane == 4) reinterpret_cast<uint32_t*>(p.blob + p.lay.off_out_ptr)[tile + 1u] = out_base + row_cnt;
-        if (tile == 0u && lane == 5) reinterpret_cast<uint32_t*>(p.blob + p.lay.off_word_off)[0] = 0u;
-        if (tile == 0u && lane == 6) reinterpret_cast<uint32_t*>(p.blob + p.lay.off_out_ptr)[0] = 0u;
+        // the token's fields
+        if (lane == 3u) field_val += word_off;
+        if (lane == 4u) field_val += out_base;
+        if (field) *reinterpret_cast<uint32_t*>(p.blob + field_off) = field_val;
+        if (lane == 0) reinterpret_cast<uint8_t*>(p.blob + p.lay.off_bits)[tile] = static_cast<uint8_t>(bstar8);
         if (row_cnt != 0u) {
           uint32_t* o_outl = reinterpret_cast<uint32_t*>(p.blob + p.lay.off_outl);
           bool overflow = false;
-          if (m.heavy != 0u) {
+          if (short_list) {
+            const unsigned long long at0 = static_cast<unsigned long long>(out_base) + lane, at1 = at0 + 32ull;
+            if (lane < row_cnt) {
+              if (at0 < p.lay.outlier_capacity) {
+                o_outl[at0] = e0;
+              } else {
+                overflow = true;
+              }
+            }
+            if (lane + 32u < row_cnt) {
+              if (at1 < p.lay.outlier_capacity) {
+                o_outl[at1] = e1;
+              } else {
+                overflow = true;
+              }
+            }
+          } else if (heavy != 0u) {
             // the compute threads write this row's entries: tell them where
             if (lane == 0) {
               sh.heavy_base = out_base;
