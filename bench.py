@@ -48,10 +48,10 @@ FALLBACK_HBM_GBS = 6650.0
 # under profiles/, keyed by kernel; each entry is valid only for the kernel source it was taken on
 # (sha256 of the .cu file) and is scaled by tokens when the capture ran a smaller case.
 NCU_TRAFFIC = {
-    "encode": {"sha256": "42168581e65cf70bb78cdd0260f5eb26b63c60ed90c8068790be670d6602c1d0",
-               "bytes_per_token": (134298368 + 35415296) / 8192, "hidden": 8192, "dtype": "bf16"},
+    "encode": {"sha256": "9f369b6f8da4de1c72cb24bcbfb7c5107516207da5c4a319645bfc4adce7f0c5",
+               "bytes_per_token": (134320896 + 35652096) / 8192, "hidden": 8192, "dtype": "bf16"},
     "decode": {"sha256": "3c9060c47b64da8ccfe6b7343d305c20c49b4fd14c9beccf2be4a0df2b8ceb1a",
-               "bytes_per_token": (68653056 + 76135680) / 8192, "hidden": 8192, "dtype": "bf16"},
+               "bytes_per_token": (68654336 + 79920128) / 8192, "hidden": 8192, "dtype": "bf16"},
 }
 KERNEL_NAMES = {"encode": "encode_pipe_kernel (encode_rows_kernel for few or very long rows)", "decode": "decode_kernel"}
 
